@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of the FLARE token mixer on B200: one step = one flare_forward over one batch of synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is whole-job tokens/s with inputs resident in HBM; `e2e` is the same
+metric through flare_forward_host with pinned host buffers (host<->device copies inside the timed region);
+`roofline` describes the slower of the two main kernels (encode, decode) against the measured peak;
+`cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.  With N > 1 every rank runs
+the same workload on its own batch (weak scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2508_12594_b200 import workloads  # noqa: E402
+
+METRIC = "FLARE fwd tokens/sec at N=1M on 1 B200"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def get_workload(name: str) -> workloads.Workload:
+    if name in workloads.CONFIGS:
+        return workloads.CONFIGS[name]
+    if name.startswith("sweep_N"):
+        n, m = name[len("sweep_N"):].split("_M")
+        return workloads.sweep_point(int(n), int(m))
+    raise SystemExit(f"unknown workload {name}")
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w: workloads.Workload, inp, sample_tokens: int):
+    """Time the CPU oracle (as it stands) on the first `sample_tokens` tokens of every batch item."""
+    from oracle import flare_oracle
+    flare_oracle.build()
+    n = min(w.N, sample_tokens)
+    Q = inp.Q.double().numpy()
+    K = inp.K[:, :n].double().numpy()
+    V = inp.V[:, :n].double().numpy()
+    mask = None if inp.key_mask is None else inp.key_mask[:, :n].numpy()
+    t0 = time.perf_counter()
+    flare_oracle.forward(Q, K, V, key_mask=mask, scale=w.scale)
+    dt = time.perf_counter() - t0
+    return w.B * n / dt, dt, n, flare_oracle.max_threads()
+
+
+def run_reference(args, w):
+    """The reference arm: the oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = workloads.make_inputs(w.with_(N=min(w.N, args.ref_tokens)))
+    times, cores, n = [], 1, 0
+    for i in range(args.warmup + args.steps):
+        v, dt, n, cores = oracle_sample(w.with_(N=inp.K.shape[1]), inp, args.ref_tokens)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = w.B * n / (ms / 1e3)
+    sample = f"first {n} tokens of each of {w.B} batch item(s), all {w.H} heads, M={w.M}, D={w.D}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "M": w.M, "D": w.D, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="mesh3d_1m")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens per batch item in the oracle sample")
+    ap.add_argument("--ref-tokens", type=int, default=16384)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = get_workload(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, w)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2508_12594_b200 import flare
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank draws its own batch (weak scaling): same recipe, rank-dependent seed
+    wr = w.with_(seed=w.seed + 1000 * rank)
+    inp = workloads.make_inputs(wr)
+    Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
+    mask = None if inp.key_mask is None else inp.key_mask.cuda()
+    desc = flare.make_desc(Q, K, w.scale)
+    ws = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    Y = torch.empty_like(K)
+    Z = torch.empty(w.B, w.H, w.M, w.D, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+    e = 4 if w.dtype == "f32" else 2
+    tensor_bytes = w.B * w.N * w.H * w.D * e
+    l2_note = "inputs larger than L2" if 3 * tensor_bytes > 2 * 126e6 else "L2 flushed between steps"
+    flush = None if 3 * tensor_bytes > 2 * 126e6 else torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def step():
+        if flush is not None:
+            flush.zero_()
+        flare.flare_forward(desc, Q, K, V, mask, Y, Z, None, None, ws, stream)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    if flush is None:
+        ev[0].record(stream)
+        for _ in range(args.steps):
+            step()
+        ev[1].record(stream)
+        barrier()
+        ms_total = ev[0].elapsed_time(ev[1])
+    else:  # time each step on its own so the flush stays outside
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in evs:
+            flush.zero_()
+            a.record(stream)
+            flare.flare_forward(desc, Q, K, V, mask, Y, Z, None, None, ws, stream)
+            b.record(stream)
+        barrier()
+        ms_total = sum(a.elapsed_time(b) for a, b in evs)
+    # per-stage durations (encode incl. merge, decode), same inputs, events on the launching stream
+    wse = flare.alloc_workspace(desc, flare.OP_ENCODE)
+    stage_ms = {}
+    for name, fn in (("encode", lambda: flare.flare_encode(desc, Q, K, V, mask, Z, None, wse, stream)),
+                     ("decode", lambda: flare.flare_decode(desc, Q, K, Z, Y, None, stream))):
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in pairs:
+            if flush is not None:
+                flush.zero_()
+            a.record(stream); fn(); b.record(stream)
+        torch.cuda.synchronize()
+        stage_ms[name] = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)
+    clocks = sampler.stop() if rank == 0 else None
+    flare.flare_check(ws)
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = world * w.tokens / (ms_step / 1e3)
+
+    # end to end: pinned host buffers in, pinned host buffer out, through flare_forward_host
+    hQ, hK, hV = inp.Q.pin_memory(), inp.K.pin_memory(), inp.V.pin_memory()
+    hmask = None if inp.key_mask is None else inp.key_mask.pin_memory()
+    hY = torch.empty_like(inp.K).pin_memory()
+    dQ, dK, dV, dY = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V), torch.empty_like(K)
+    dmask = None if mask is None else torch.empty_like(mask)
+    for _ in range(2):
+        flare.flare_forward_host(desc, hQ, hK, hV, hmask, hY, dQ, dK, dV, dmask, dY, ws, stream)
+    barrier()
+    ev[0].record(stream)
+    for _ in range(args.e2e_steps):
+        flare.flare_forward_host(desc, hQ, hK, hV, hmask, hY, dQ, dK, dV, dmask, dY, ws, stream)
+    ev[1].record(stream)
+    barrier()
+    t = torch.tensor([ev[0].elapsed_time(ev[1])], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item()) / args.e2e_steps
+    h2d = 2 * tensor_bytes + w.H * w.M * w.D * e + (0 if mask is None else w.B * w.N)
+    e2e = {"value": world * w.tokens / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": tensor_bytes, "ms_per_step": e2e_ms}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    # Roofline of the slower main kernel.  Per stage and head the contraction work is 4*N*M*D FLOP (scores and
+    # value contraction); the bytes are K and V read (encode) or K read and Y written (decode), plus Q_lat.
+    flops_stage = 4.0 * w.B * w.H * w.N * w.M * w.D
+    bytes_stage = 2.0 * tensor_bytes + w.H * w.M * w.D * e
+    dom = max(stage_ms, key=stage_ms.get)
+    t_dom = stage_ms[dom] / 1e3
+    tensor_peak = peaks["bf16_tflops"] * (0.5 if w.dtype == "f32" else 1.0)
+    t_tensor, t_hbm = flops_stage / (tensor_peak * 1e12), bytes_stage / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        roof = {"bound": "tensor", "achieved": flops_stage / t_dom / 1e12, "peak": tensor_peak, "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": bytes_stage / t_dom / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof.update({"traffic": None, "kernel": dom, "kernel_ms": stage_ms[dom], "peak_kind": peak_kind,
+                 "stage_ms": stage_ms, "exp_per_s": w.B * w.H * w.N * w.M / t_dom})
+    # whole forward against the stated roofline: slower of 8*B*H*N*M*D FLOP at tensor peak and K, V, Q_lat, Y once
+    fwd_t = max(2 * flops_stage / (tensor_peak * 1e12), (3 * tensor_bytes + w.H * w.M * w.D * e) / (peaks["hbm_gbs"] * 1e9))
+    roof["forward_frac_of_stated_roofline"] = fwd_t / (ms_step / 1e3)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "M": w.M, "D": w.D, "scale": w.scale,
+                   "l2": l2_note, "parallelism": f"replicas x{world}"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roof,
+    }
+    if not args.no_cpu_baseline:
+        v, dt, n, cores = oracle_sample(w, inp, args.cpu_tokens)
+        out["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                               "sample": f"first {n} tokens of each of {w.B} batch item(s), all heads, {dt:.1f} s"}
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

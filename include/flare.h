@@ -1,0 +1,144 @@
+/*
+ * libflare -- C ABI of the FLARE token mixer for NVIDIA B200 (sm_100a).
+ *
+ * The operator (paper Section 3.2): for every batch item b and head h, M latent queries attend over the N
+ * tokens (encode), then the N tokens attend back over the M latents with queries and keys swapped and the
+ * latent sequence as values (decode):
+ *
+ *     Z[b,h]  = softmax_rows(scale * Q[h] K[b,:,h]^T) V[b,:,h]        (encode equation; M x D)
+ *     Y[b,:,h] = softmax_rows(scale * K[b,:,h] Q[h]^T) Z[b,h]         (decode equation; N x D)
+ *
+ * The paper fixes scale = 1 in both stages; it is a parameter here.  No M x N or N x N matrix is ever
+ * written to memory.
+ *
+ * Layouts (all contiguous, row-major, innermost index last):
+ *     Q_lat            [H, M, D]      dtype      latent queries, shared by all batch items
+ *     K, V, Y, dY, dK, dV [B, N, H, D] dtype      token-major
+ *     Z, dZ            [B, H, M, D]   float32    latent sequence
+ *     lse_enc          [B, H, M]      float32    log sum_n exp(score) over valid tokens (-inf if none)
+ *     lse_dec          [B, N, H]      float32    log sum_m exp(score)
+ *     key_mask         [B, N]         uint8      1 = valid token, 0 = padding; NULL = all valid
+ *     dQ_lat           [H, M, D]      float32    summed over the batch
+ *
+ * Padding (not in the paper): a masked token takes no part in the encode softmax; decode is evaluated for
+ * every token.  A batch item with no valid token gets Z = 0, lse_enc = -inf.
+ *
+ * Pointers and ownership: unless a function says "host", every pointer is a DEVICE pointer to memory owned
+ * by the caller, 16-byte aligned; the library never allocates, frees or keeps them.  Calls enqueue work on
+ * `stream` and return without synchronising; outputs are overwritten, never accumulated into.  Two calls may
+ * run concurrently on different streams only with different workspaces.  Results are bitwise reproducible
+ * for a fixed descriptor on a fixed device.
+ *
+ * Supported shapes: D in {8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 512.
+ * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation.
+ *
+ * Every entry point returns a flare_status_t; nothing is thrown, nothing is printed.
+ */
+#ifndef FLARE_H_
+#define FLARE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *flare_stream_t; /* a cudaStream_t */
+
+typedef enum {
+    FLARE_OK = 0,
+    FLARE_ERR_INVALID_ARG = 1,         /* null pointer, non-positive size, misaligned pointer, non-finite scale */
+    FLARE_ERR_UNSUPPORTED = 2,         /* shape or dtype outside the supported set */
+    FLARE_ERR_WORKSPACE_TOO_SMALL = 3, /* workspace_bytes < flare_workspace_bytes(desc, op) */
+    FLARE_ERR_ARCH = 4,                /* current device is not compute capability 10.x */
+    FLARE_ERR_CUDA = 5,                /* a CUDA call or launch failed; flare_last_cuda_error() has the text */
+    FLARE_ERR_TIMEOUT = 6              /* a bounded device-side wait gave up (reported by flare_check) */
+} flare_status_t;
+
+enum { FLARE_DTYPE_F32 = 0, FLARE_DTYPE_BF16 = 1 };
+enum { FLARE_OP_ENCODE = 0, FLARE_OP_DECODE = 1, FLARE_OP_FORWARD = 2, FLARE_OP_BACKWARD = 3 };
+
+typedef struct {
+    int32_t B, H, N, M, D; /* batch, heads, tokens, latents per head, head width */
+    int32_t dtype;         /* FLARE_DTYPE_* : element type of Q_lat, K, V, Y, dY, dK, dV */
+    float scale;           /* multiplies every q.k score; the paper uses 1.0f */
+} flare_desc_t;
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int flare_version(void);
+
+/* Static text for a status code (never NULL). */
+const char *flare_status_string(int status);
+
+/* Text of the last CUDA error seen by this thread inside the library ("" if none).  Host pointer. */
+const char *flare_last_cuda_error(void);
+
+/*
+ * Bytes of scratch `workspace` the given operation needs for `desc` on the current device (0 for an invalid
+ * or unsupported descriptor).  Encode writes per-split partial results (running maximum, sum and
+ * un-normalised latent rows) there: O(splits * B * H * M * (D + 2)) floats, never anything of size N x M.
+ */
+size_t flare_workspace_bytes(const flare_desc_t *desc, int op);
+
+/* Number of partial results per (b, h, latent) that encode produces and the merge step combines. */
+int flare_encode_partials(const flare_desc_t *desc);
+
+/*
+ * Encode (Section 3.2, encode equation; per-latent sum of the design-principles appendix):
+ * Z and, if lse_enc != NULL, lse_enc.  Split over N: every CTA keeps a running maximum and sum per latent
+ * (online softmax) over its token range; a second kernel merges the splits by log-sum-exp.
+ */
+int flare_encode(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
+                 const uint8_t *key_mask, float *Z, float *lse_enc, void *workspace, size_t workspace_bytes,
+                 flare_stream_t stream);
+
+/*
+ * Decode (Section 3.2, decode equation; per-token sum of the design-principles appendix):
+ * Y and, if lse_dec != NULL, lse_dec, from K, Q_lat and a latent sequence Z.  Needs no workspace.
+ */
+int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *Z, void *Y,
+                 float *lse_dec, flare_stream_t stream);
+
+/*
+ * The whole mixer (the paper's two-call listing in Section 3.2): encode, merge, decode on one stream.
+ * Z, lse_enc, lse_dec may each be NULL; a NULL Z lives in the workspace.
+ */
+int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
+                  const uint8_t *key_mask, void *Y, float *Z, float *lse_enc, float *lse_dec, void *workspace,
+                  size_t workspace_bytes, flare_stream_t stream);
+
+/*
+ * Backward of flare_forward.  The paper times a backward pass but does not write it out; this is the chain
+ * rule applied to the two equations above (W_enc, W_dec the two softmax matrices, recomputed tile by tile):
+ *     dZ = W_dec^T dY;  dV = W_enc^T dZ;
+ *     dS[m,n] = W_dec[n,m] (dY_n.Z_m - dY_n.Y_n) + W_enc[m,n] (dZ_m.V_n - dZ_m.Z_m);
+ *     dQ_lat = scale * sum_b dS K;  dK = scale * dS^T Q_lat.
+ * Z, lse_enc, lse_dec are the ones flare_forward wrote; Y is its output.
+ */
+int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
+                   const uint8_t *key_mask, const void *Y, const void *dY, const float *Z, const float *lse_enc,
+                   const float *lse_dec, float *dQ_lat, void *dK, void *dV, void *workspace,
+                   size_t workspace_bytes, flare_stream_t stream);
+
+/*
+ * flare_forward for callers whose tensors live in HOST memory (pinned memory makes the copies asynchronous).
+ * Copies Q_lat, K, V (and key_mask if not NULL) from the host pointers into the caller's device staging
+ * buffers dQ_lat, dK, dV, dmask, runs flare_forward into dY, and copies Y back to hY, all on `stream`.
+ * hQ_lat, hK, hV, hmask, hY are host pointers; everything else is a device pointer.
+ */
+int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void *hK, const void *hV,
+                       const uint8_t *hmask, void *hY, void *dQ_lat, void *dK, void *dV, uint8_t *dmask, void *dY,
+                       void *workspace, size_t workspace_bytes, flare_stream_t stream);
+
+/*
+ * After the stream has been synchronised: FLARE_OK, or FLARE_ERR_TIMEOUT if a kernel of the last call that
+ * used `workspace` gave up on a bounded wait (its outputs are then undefined).  Reads one word from the
+ * workspace with a blocking copy.
+ */
+int flare_check(const void *workspace, flare_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLARE_H_ */

@@ -1,0 +1,291 @@
+// Host side of libflare: argument checks, launch plans, kernel launches.  See include/flare.h for the contract.
+#include "../../include/flare.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "flare_common.cuh"
+#include "flare_simt.cuh"
+
+using namespace flare;
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char *what) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+    return FLARE_ERR_CUDA;
+}
+
+#define FLARE_CUDA(call)                                      \
+    do {                                                      \
+        cudaError_t e__ = (call);                             \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+struct DeviceInfo {
+    int checked = 0;  // 0 = not yet, 1 = ok, -1 = wrong arch, -2 = no device
+    int sms = 148;
+};
+DeviceInfo g_dev[64];
+
+// Properties of the current device (cached per ordinal).  Without a device the plan falls back to 148 SMs so
+// that size queries still answer.
+const DeviceInfo &device_info(int *ordinal_out = nullptr) {
+    static DeviceInfo none{-2, 148};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return none;
+    }
+    if (ordinal_out) *ordinal_out = dev;
+    DeviceInfo &d = g_dev[dev];
+    if (d.checked == 0) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return none;
+        }
+        d.sms = sms > 0 ? sms : 148;
+        d.checked = (major == 10) ? 1 : -1;
+    }
+    return d;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_desc(const flare_desc_t *d) {
+    if (d == nullptr) return FLARE_ERR_INVALID_ARG;
+    if (d->B <= 0 || d->H <= 0 || d->N <= 0 || d->M <= 0 || d->D <= 0) return FLARE_ERR_INVALID_ARG;
+    if (!std::isfinite(d->scale)) return FLARE_ERR_INVALID_ARG;
+    if (d->dtype != FLARE_DTYPE_F32 && d->dtype != FLARE_DTYPE_BF16) return FLARE_ERR_UNSUPPORTED;
+    if (d->D != 8 && d->D != 16 && d->D != 32 && d->D != 64) return FLARE_ERR_UNSUPPORTED;
+    if (d->dtype == FLARE_DTYPE_BF16 && (d->M % 16 != 0 || d->M < 16 || d->M > 512)) return FLARE_ERR_UNSUPPORTED;
+    if ((long)d->B * d->N > (1L << 31) - 1 || d->H > 65535 || d->B > 65535) return FLARE_ERR_UNSUPPORTED;
+    return FLARE_OK;
+}
+
+// Launch plan of the CUDA-core encode: LM latents x G token groups per block, `splits` blocks along N.
+struct SimtPlan {
+    int LM, G, splits, chunk, P;
+};
+
+SimtPlan simt_plan(const flare_desc_t *d, int sms) {
+    SimtPlan p;
+    p.LM = 1;
+    while (p.LM < d->M && p.LM < kSimtThreads) p.LM *= 2;
+    p.G = kSimtThreads / p.LM;
+    long bh = (long)d->B * d->H;
+    long want = (4L * sms + bh - 1) / bh;                  // about four blocks per SM in total
+    long most = (d->N + 255) / 256;                        // at least 256 tokens per block
+    long s = want < most ? want : most;
+    if (s < 1) s = 1;
+    p.chunk = (int)((d->N + s - 1) / s);
+    p.chunk = (p.chunk + kSimtTileN - 1) / kSimtTileN * kSimtTileN;
+    p.splits = (d->N + p.chunk - 1) / p.chunk;
+    p.P = p.splits * p.G;
+    return p;
+}
+
+int partials_for(const flare_desc_t *d, int sms) { return simt_plan(d, sms).P; }
+
+template <typename T>
+int launch_encode_simt(const flare_desc_t *d, const SimtPlan &p, const void *Q, const void *K, const void *V,
+                       const uint8_t *mask, float *pm, float *pl, float *pacc, cudaStream_t st) {
+    dim3 grid(p.splits, d->H, d->B), block(kSimtThreads);
+#define FLARE_CASE(DD)                                                                                          \
+    case DD:                                                                                                    \
+        encode_simt_kernel<T, DD><<<grid, block, 0, st>>>((const T *)Q, (const T *)K, (const T *)V, mask, pm, pl, \
+                                                          pacc, d->B, d->H, d->N, d->M, p.LM, p.chunk, d->scale); \
+        break;
+    switch (d->D) {
+        FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
+        default: return FLARE_ERR_UNSUPPORTED;
+    }
+#undef FLARE_CASE
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+template <typename T>
+int launch_decode_simt(const flare_desc_t *d, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
+                       cudaStream_t st) {
+    dim3 grid((d->N + kDecodeSimtThreads - 1) / kDecodeSimtThreads, d->H, d->B), block(kDecodeSimtThreads);
+#define FLARE_CASE(DD)                                                                                            \
+    case DD:                                                                                                      \
+        decode_simt_kernel<T, DD><<<grid, block, 0, st>>>((const T *)Q, (const T *)K, Z, (T *)Y, lse_dec, d->B, d->H, \
+                                                          d->N, d->M, d->scale);                                  \
+        break;
+    switch (d->D) {
+        FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
+        default: return FLARE_ERR_UNSUPPORTED;
+    }
+#undef FLARE_CASE
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+int require_device() {
+    const DeviceInfo &di = device_info();
+    if (di.checked == -2) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "no CUDA device");
+        return FLARE_ERR_CUDA;
+    }
+    if (di.checked != 1) return FLARE_ERR_ARCH;
+    return FLARE_OK;
+}
+
+int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void *V, const uint8_t *mask, float *Z,
+                float *lse_enc, void *ws, cudaStream_t st) {
+    const DeviceInfo &di = device_info();
+    const long rows = (long)d->B * d->H * d->M;
+    SimtPlan p = simt_plan(d, di.sms);
+    WorkspaceLayout w = make_layout(p.P, rows, d->D, false);
+    char *base = static_cast<char *>(ws);
+    float *pm = reinterpret_cast<float *>(base + w.part_m);
+    float *pl = reinterpret_cast<float *>(base + w.part_l);
+    float *pacc = reinterpret_cast<float *>(base + w.part_acc);
+    FLARE_CUDA(cudaMemsetAsync(base, 0, kHeaderBytes, st));
+    int rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)
+                                           : launch_encode_simt<__nv_bfloat16>(d, p, Q, K, V, mask, pm, pl, pacc, st);
+    if (rc != FLARE_OK) return rc;
+    const long total = rows * d->D;
+    merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(pm, pl, pacc, Z, lse_enc, p.P, rows, d->D);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
+                cudaStream_t st) {
+    return (d->dtype == FLARE_DTYPE_F32) ? launch_decode_simt<float>(d, Q, K, Z, Y, lse_dec, st)
+                                         : launch_decode_simt<__nv_bfloat16>(d, Q, K, Z, Y, lse_dec, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int flare_version(void) { return 100; }
+
+const char *flare_status_string(int status) {
+    switch (status) {
+        case FLARE_OK: return "ok";
+        case FLARE_ERR_INVALID_ARG: return "invalid argument";
+        case FLARE_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case FLARE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case FLARE_ERR_ARCH: return "device is not compute capability 10.x";
+        case FLARE_ERR_CUDA: return "CUDA error";
+        case FLARE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+const char *flare_last_cuda_error(void) { return g_cuda_error; }
+
+int flare_encode_partials(const flare_desc_t *desc) {
+    if (check_desc(desc) != FLARE_OK) return 0;
+    return partials_for(desc, device_info().sms);
+}
+
+size_t flare_workspace_bytes(const flare_desc_t *desc, int op) {
+    if (check_desc(desc) != FLARE_OK) return 0;
+    const long rows = (long)desc->B * desc->H * desc->M;
+    switch (op) {
+        case FLARE_OP_ENCODE: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, false).total;
+        case FLARE_OP_DECODE: return kHeaderBytes;
+        case FLARE_OP_FORWARD: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, true).total;
+        case FLARE_OP_BACKWARD: return 0;
+        default: return 0;
+    }
+}
+
+int flare_encode(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,
+                 float *Z, float *lse_enc, void *workspace, size_t workspace_bytes, flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    if (!Q_lat || !K || !V || !Z || !workspace) return FLARE_ERR_INVALID_ARG;
+    if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(V) || !aligned16(Z) || !aligned16(workspace) ||
+        (lse_enc && !aligned16(lse_enc)))
+        return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    if (workspace_bytes < flare_workspace_bytes(desc, FLARE_OP_ENCODE)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    return encode_impl(desc, Q_lat, K, V, key_mask, Z, lse_enc, workspace, (cudaStream_t)stream);
+}
+
+int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *Z, void *Y, float *lse_dec,
+                 flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    if (!Q_lat || !K || !Z || !Y) return FLARE_ERR_INVALID_ARG;
+    if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(Z) || !aligned16(Y) || (lse_dec && !aligned16(lse_dec)))
+        return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, (cudaStream_t)stream);
+}
+
+int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,
+                  void *Y, float *Z, float *lse_enc, float *lse_dec, void *workspace, size_t workspace_bytes,
+                  flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    if (!Q_lat || !K || !V || !Y || !workspace) return FLARE_ERR_INVALID_ARG;
+    if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(V) || !aligned16(Y) || !aligned16(workspace) ||
+        (Z && !aligned16(Z)) || (lse_enc && !aligned16(lse_enc)) || (lse_dec && !aligned16(lse_dec)))
+        return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    if (workspace_bytes < flare_workspace_bytes(desc, FLARE_OP_FORWARD)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    if (Z == nullptr) {
+        const long rows = (long)desc->B * desc->H * desc->M;
+        WorkspaceLayout w = make_layout(partials_for(desc, device_info().sms), rows, desc->D, true);
+        Z = reinterpret_cast<float *>(static_cast<char *>(workspace) + w.z);
+    }
+    rc = encode_impl(desc, Q_lat, K, V, key_mask, Z, lse_enc, workspace, (cudaStream_t)stream);
+    if (rc != FLARE_OK) return rc;
+    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, (cudaStream_t)stream);
+}
+
+int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,
+                   const void *Y, const void *dY, const float *Z, const float *lse_enc, const float *lse_dec,
+                   float *dQ_lat, void *dK, void *dV, void *workspace, size_t workspace_bytes,
+                   flare_stream_t stream) {
+    (void)Q_lat; (void)K; (void)V; (void)key_mask; (void)Y; (void)dY; (void)Z; (void)lse_enc; (void)lse_dec;
+    (void)dQ_lat; (void)dK; (void)dV; (void)workspace; (void)workspace_bytes; (void)stream;
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    return FLARE_ERR_UNSUPPORTED;
+}
+
+int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void *hK, const void *hV,
+                       const uint8_t *hmask, void *hY, void *dQ_lat, void *dK, void *dV, uint8_t *dmask, void *dY,
+                       void *workspace, size_t workspace_bytes, flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    if (!hQ_lat || !hK || !hV || !hY || !dQ_lat || !dK || !dV || !dY || (hmask && !dmask)) return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t e = desc->dtype == FLARE_DTYPE_F32 ? 4 : 2;
+    const size_t qb = (size_t)desc->H * desc->M * desc->D * e;
+    const size_t tb = (size_t)desc->B * desc->N * desc->H * desc->D * e;
+    FLARE_CUDA(cudaMemcpyAsync(dQ_lat, hQ_lat, qb, cudaMemcpyHostToDevice, st));
+    FLARE_CUDA(cudaMemcpyAsync(dK, hK, tb, cudaMemcpyHostToDevice, st));
+    FLARE_CUDA(cudaMemcpyAsync(dV, hV, tb, cudaMemcpyHostToDevice, st));
+    if (hmask) FLARE_CUDA(cudaMemcpyAsync(dmask, hmask, (size_t)desc->B * desc->N, cudaMemcpyHostToDevice, st));
+    rc = flare_forward(desc, dQ_lat, dK, dV, hmask ? dmask : nullptr, dY, nullptr, nullptr, nullptr, workspace,
+                       workspace_bytes, stream);
+    if (rc != FLARE_OK) return rc;
+    FLARE_CUDA(cudaMemcpyAsync(hY, dY, tb, cudaMemcpyDeviceToHost, st));
+    return FLARE_OK;
+}
+
+int flare_check(const void *workspace, flare_stream_t stream) {
+    if (!workspace) return FLARE_ERR_INVALID_ARG;
+    uint32_t words[2] = {0, 0};
+    FLARE_CUDA(cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    FLARE_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return words[0] == 0 ? FLARE_OK : FLARE_ERR_TIMEOUT;
+}
+
+}  // extern "C"

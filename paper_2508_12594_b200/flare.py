@@ -1,0 +1,207 @@
+"""Python binding of libflare: the same entry points as ``include/flare.h``, argument marshalling only.
+
+Every step of the mixer runs in the library's CUDA kernels.  PyTorch is used for device memory and streams:
+the functions take torch tensors, check layout and dtype, and pass raw pointers.  There is no CPU fallback:
+if ``libflare.so`` is missing or cannot be loaded the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libflare.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(7)
+DTYPE_F32, DTYPE_BF16 = 0, 1
+OP_ENCODE, OP_DECODE, OP_FORWARD, OP_BACKWARD = range(4)
+
+
+class FlareDesc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32), ("M", ctypes.c_int32),
+                ("D", ctypes.c_int32), ("dtype", ctypes.c_int32), ("scale", ctypes.c_float)]
+
+
+class FlareError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        lib = _lib_or_none()
+        text = lib.flare_status_string(status).decode() if lib else str(status)
+        detail = lib.flare_last_cuda_error().decode() if lib and status == ERR_CUDA else ""
+        super().__init__(f"{where}: {text}" + (f" ({detail})" if detail else ""))
+        self.status = status
+
+
+_lib = None
+
+_vp, _sz = ctypes.c_void_p, ctypes.c_size_t
+_dp = ctypes.POINTER(FlareDesc)
+_SIGNATURES = {
+    "flare_version": (ctypes.c_int, []),
+    "flare_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "flare_last_cuda_error": (ctypes.c_char_p, []),
+    "flare_workspace_bytes": (_sz, [_dp, ctypes.c_int]),
+    "flare_encode_partials": (ctypes.c_int, [_dp]),
+    "flare_encode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "flare_decode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "flare_forward": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 14 + [_sz, _vp]),
+    "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
+    "flare_check": (ctypes.c_int, [_vp, _vp]),
+}
+
+
+def _lib_or_none():
+    return _lib
+
+
+def load():
+    """Load libflare.so (once).  Raises if the CUDA extension has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2508_12594_b200.build`")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def exported_symbols():
+    return list(_SIGNATURES)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def make_desc(Q: torch.Tensor, K: torch.Tensor, scale: float = 1.0) -> FlareDesc:
+    H, M, D = Q.shape
+    B, N, H2, D2 = K.shape
+    if (H2, D2) != (H, D):
+        raise ValueError("Q_lat [H,M,D] and K [B,N,H,D] disagree")
+    return FlareDesc(B, H, N, M, D, _dtype_code(K), float(scale))
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, shape=None, cuda=True):
+    if t is None:
+        return None
+    if cuda and not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {t.dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _raise(rc: int, where: str):
+    if rc != OK:
+        raise FlareError(rc, where)
+
+
+def flare_version() -> int:
+    return load().flare_version()
+
+
+def flare_workspace_bytes(desc: FlareDesc, op: int) -> int:
+    return int(load().flare_workspace_bytes(ctypes.byref(desc), op))
+
+
+def flare_encode_partials(desc: FlareDesc) -> int:
+    return int(load().flare_encode_partials(ctypes.byref(desc)))
+
+
+def alloc_workspace(desc: FlareDesc, op: int, device="cuda") -> torch.Tensor:
+    n = flare_workspace_bytes(desc, op)
+    if n == 0:
+        raise FlareError(ERR_UNSUPPORTED, "flare_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def flare_encode(desc, Q, K, V, key_mask, Z, lse_enc, workspace, stream=None):
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    rc = load().flare_encode(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, (B, N, H, D)),
+                             _ptr(V, dt, (B, N, H, D)), _ptr(key_mask, torch.uint8, (B, N)),
+                             _ptr(Z, torch.float32, (B, H, M, D)), _ptr(lse_enc, torch.float32, (B, H, M)),
+                             _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
+    _raise(rc, "flare_encode")
+
+
+def flare_decode(desc, Q, K, Z, Y, lse_dec, stream=None):
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    rc = load().flare_decode(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, (B, N, H, D)),
+                             _ptr(Z, torch.float32, (B, H, M, D)), _ptr(Y, dt, (B, N, H, D)),
+                             _ptr(lse_dec, torch.float32, (B, N, H)), _stream(stream))
+    _raise(rc, "flare_decode")
+
+
+def flare_forward(desc, Q, K, V, key_mask, Y, Z, lse_enc, lse_dec, workspace, stream=None):
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    rc = load().flare_forward(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, (B, N, H, D)),
+                              _ptr(V, dt, (B, N, H, D)), _ptr(key_mask, torch.uint8, (B, N)),
+                              _ptr(Y, dt, (B, N, H, D)), _ptr(Z, torch.float32, (B, H, M, D)),
+                              _ptr(lse_enc, torch.float32, (B, H, M)), _ptr(lse_dec, torch.float32, (B, N, H)),
+                              _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
+    _raise(rc, "flare_forward")
+
+
+def flare_backward(desc, Q, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, workspace, stream=None):
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    tok = (B, N, H, D)
+    rc = load().flare_backward(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, tok), _ptr(V, dt, tok),
+                               _ptr(key_mask, torch.uint8, (B, N)), _ptr(Y, dt, tok), _ptr(dY, dt, tok),
+                               _ptr(Z, torch.float32, (B, H, M, D)), _ptr(lse_enc, torch.float32, (B, H, M)),
+                               _ptr(lse_dec, torch.float32, (B, N, H)), _ptr(dQ, torch.float32, (H, M, D)),
+                               _ptr(dK, dt, tok), _ptr(dV, dt, tok), _ptr(workspace, torch.uint8),
+                               workspace.numel(), _stream(stream))
+    _raise(rc, "flare_backward")
+
+
+def flare_forward_host(desc, hQ, hK, hV, hmask, hY, dQ, dK, dV, dmask, dY, workspace, stream=None):
+    """Host tensors in, host tensor out; the device tensors are the caller's staging buffers."""
+    dt = hK.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    tok = (B, N, H, D)
+    rc = load().flare_forward_host(ctypes.byref(desc), _ptr(hQ, dt, (H, M, D), cuda=False), _ptr(hK, dt, tok, cuda=False),
+                                   _ptr(hV, dt, tok, cuda=False), _ptr(hmask, torch.uint8, (B, N), cuda=False),
+                                   _ptr(hY, dt, tok, cuda=False), _ptr(dQ, dt, (H, M, D)), _ptr(dK, dt, tok),
+                                   _ptr(dV, dt, tok), _ptr(dmask, torch.uint8, (B, N)), _ptr(dY, dt, tok),
+                                   _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
+    _raise(rc, "flare_forward_host")
+
+
+def flare_check(workspace, stream=None):
+    _raise(load().flare_check(_ptr(workspace, torch.uint8), _stream(stream)), "flare_check")
+
+
+def forward(Q, K, V, key_mask=None, scale=1.0, want_stats=False, stream=None):
+    """Convenience: allocate outputs and workspace with torch, call flare_forward, return Y (and Z, lse's)."""
+    desc = make_desc(Q, K, scale)
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    ws = alloc_workspace(desc, OP_FORWARD, K.device)
+    Y = torch.empty_like(K)
+    Z = torch.empty(B, H, M, D, dtype=torch.float32, device=K.device)
+    le = torch.empty(B, H, M, dtype=torch.float32, device=K.device)
+    ld = torch.empty(B, N, H, dtype=torch.float32, device=K.device)
+    flare_forward(desc, Q, K, V, key_mask, Y, Z, le, ld, ws, stream)
+    return (Y, Z, le, ld) if want_stats else Y

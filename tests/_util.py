@@ -1,0 +1,72 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C-ABI binding, run the oracle on the
+same stored input values, compare with the relative-to-RMS bound."""
+import numpy as np
+import torch
+
+from paper_2508_12594_b200 import flare
+
+# max |err| <= tol * RMS(reference), per tensor: 1e-5 for float32 inputs, 2e-2 for bfloat16 inputs with float32
+# accumulation (three bf16 roundings of relative size 2^-9 each: the softmax weights, Z and the stored Y).
+TOL = {"f32": 1e-5, "bf16": 2e-2}
+
+
+def rel_err(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    return float(np.abs(got - ref).max()) / max(rms, 1e-300)
+
+
+def to_np64(t):
+    return None if t is None else t.double().cpu().numpy()
+
+
+def dev(t):
+    return None if t is None else t.cuda()
+
+
+def gpu_forward(inp, scale=1.0, canary=False):
+    """flare_forward on cuda:0.  With canary=True the outputs sit inside larger buffers whose margins must stay
+    untouched (checked here).  Returns numpy float64 dict(Y, Z, lse_enc, lse_dec)."""
+    Q, K, V, mask = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask)
+    desc = flare.make_desc(Q, K, scale)
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    ws = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    pad = 64 if canary else 0
+
+    def padded(shape, dtype, fill):
+        n = int(np.prod(shape))
+        buf = torch.full((n + 2 * pad,), fill, dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + n].view(*shape)
+
+    Yb, Y = padded((B, N, H, D), K.dtype, 777.0)
+    Zb, Z = padded((B, H, M, D), torch.float32, 777.0)
+    leb, le = padded((B, H, M), torch.float32, 777.0)
+    ldb, ld = padded((B, N, H), torch.float32, 777.0)
+    if pad % 8 != 0:
+        raise AssertionError("canary margin must keep 16-byte alignment")
+    flare.flare_forward(desc, Q, K, V, mask, Y, Z, le, ld, ws)
+    torch.cuda.synchronize()
+    flare.flare_check(ws)
+    if canary:
+        for buf in (Yb, Zb, leb, ldb):
+            assert (buf[:pad] == 777.0).all() and (buf[-pad:] == 777.0).all(), "write outside an output buffer"
+    return dict(Y=to_np64(Y), Z=to_np64(Z), lse_enc=to_np64(le), lse_dec=to_np64(ld))
+
+
+def oracle_forward(oracle, inp, scale=1.0):
+    mask = None if inp.key_mask is None else inp.key_mask.numpy()
+    return oracle.forward(to_np64(inp.Q), to_np64(inp.K), to_np64(inp.V), key_mask=mask, scale=scale)
+
+
+def assert_forward_close(got, ref, dtype, what=""):
+    tol = TOL[dtype]
+    for name in ("Z", "Y"):
+        e = rel_err(got[name], ref[name])
+        assert e <= tol, f"{what} {name}: max|err|/RMS = {e:.3e} > {tol}"
+    for name in ("lse_enc", "lse_dec"):
+        fin = np.isfinite(ref[name])
+        assert np.array_equal(np.isneginf(got[name]), np.isneginf(ref[name])), f"{what} {name}: -inf pattern"
+        if fin.any():
+            err = np.abs(got[name][fin] - ref[name][fin]).max()
+            assert err <= (1e-4 if dtype == "f32" else 2e-2), f"{what} {name}: abs err {err:.3e}"

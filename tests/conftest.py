@@ -17,3 +17,13 @@ def oracle():
     from oracle import flare_oracle
     flare_oracle.build()
     return flare_oracle
+
+
+def pytest_collection_modifyitems(config, items):
+    import torch
+    if torch.cuda.is_available():
+        return
+    skip = pytest.mark.skip(reason="no CUDA device")
+    for item in items:
+        if "gpu" in item.keywords:
+            item.add_marker(skip)

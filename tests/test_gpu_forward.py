@@ -1,0 +1,147 @@
+"""Parity of the CUDA path against the CPU oracle, element by element, through the C-ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2508_12594_b200 import flare, workloads
+from tests._util import TOL, assert_forward_close, dev, gpu_forward, oracle_forward, rel_err, to_np64
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tiny_config_fp32(oracle):
+    w = workloads.CONFIGS["tiny"]
+    inp = workloads.make_inputs(w)
+    assert_forward_close(gpu_forward(inp, canary=True), oracle_forward(oracle, inp), "f32", "tiny")
+
+
+# Shapes of the benchmark workloads at sizes the oracle finishes in seconds; N spans several tiles and ends in
+# a ragged tail.
+SCALED = [
+    workloads.CONFIGS["mesh2d"].with_(B=2, N=3001),
+    workloads.CONFIGS["padded"].with_(B=3, N=1000),
+    workloads.CONFIGS["mesh3d_1m"].with_(N=5003),
+    workloads.sweep_point(2500, 32),
+    workloads.sweep_point(2500, 128),
+    workloads.sweep_point(1300, 512),
+]
+
+
+@pytest.mark.parametrize("w", SCALED, ids=lambda w: w.name)
+@pytest.mark.parametrize("paper_scale", [True, False], ids=["s=1", "s=1/sqrtD"])
+def test_scaled_down_workloads(oracle, w, paper_scale):
+    scale = 1.0 if paper_scale else w.D ** -0.5
+    inp = workloads.make_inputs(w)
+    assert_forward_close(gpu_forward(inp, scale, canary=True), oracle_forward(oracle, inp, scale), w.dtype, w.name)
+
+
+EDGE = [
+    # B, H, N, M, D, dtype, masked_fraction
+    (1, 1, 1, 16, 16, "bf16", 0.0),
+    (1, 1, 1, 1, 8, "f32", 0.0),
+    (2, 3, 7, 16, 8, "bf16", 0.0),
+    (1, 2, 127, 48, 16, "bf16", 0.0),
+    (1, 2, 129, 64, 32, "bf16", 0.3),
+    (2, 1, 300, 256, 64, "bf16", 0.0),
+    (1, 1, 515, 512, 16, "bf16", 0.5),
+    (1, 2, 1000, 80, 32, "bf16", 0.0),
+    (3, 2, 333, 5, 32, "f32", 0.4),
+    (1, 1, 2049, 300, 64, "f32", 0.0),
+    (1, 4, 64, 1, 16, "f32", 0.0),
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=lambda c: "B{}H{}N{}M{}D{}{}m{}".format(*c))
+def test_edge_shapes(oracle, case):
+    B, H, N, M, D, dtype, mf = case
+    inp = workloads.make_random(B, H, N, M, D, dtype=dtype, seed=N + M, masked_fraction=mf, k_std=0.8)
+    assert_forward_close(gpu_forward(inp, canary=True), oracle_forward(oracle, inp), dtype, str(case))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_mask_degenerate_cases(oracle, dtype):
+    """All but one token masked; one batch item entirely masked (Z = 0, lse_enc = -inf, Y = 0)."""
+    inp = workloads.make_random(2, 2, 200, 16, 16, dtype=dtype, seed=5)
+    mask = torch.zeros(2, 200, dtype=torch.uint8)
+    mask[0, 137] = 1
+    inp.key_mask = mask
+    got, ref = gpu_forward(inp, canary=True), oracle_forward(oracle, inp)
+    assert_forward_close(got, ref, dtype, "degenerate mask")
+    assert (got["Z"][1] == 0).all() and (got["Y"][1] == 0).all() and np.isneginf(got["lse_enc"][1]).all()
+    np.testing.assert_allclose(got["Z"][0], np.broadcast_to(to_np64(inp.V)[0, 137][:, None, :], got["Z"][0].shape),
+                               rtol=1e-6)
+
+
+def test_single_latent_broadcasts_one_row(oracle):
+    inp = workloads.make_random(1, 2, 500, 1, 16, dtype="f32", seed=3)
+    got = gpu_forward(inp)
+    assert np.abs(got["Y"] - got["Y"][:, :1]).max() == 0.0
+    assert_forward_close(got, oracle_forward(oracle, inp), "f32", "M=1")
+
+
+def test_large_scores_do_not_overflow(oracle):
+    """Scores of several tens (natural units): the running maximum keeps every exponential finite."""
+    inp = workloads.make_random(1, 2, 700, 32, 32, dtype="bf16", seed=9, k_std=2.5, q_std=2.0)
+    got, ref = gpu_forward(inp), oracle_forward(oracle, inp)
+    assert np.isfinite(got["Y"]).all()
+    assert_forward_close(got, ref, "bf16", "large scores")
+
+
+@pytest.mark.parametrize("w", [workloads.CONFIGS["tiny"], workloads.CONFIGS["mesh3d_1m"].with_(N=40000)],
+                         ids=lambda w: w.name)
+def test_bitwise_reproducible(w):
+    inp = workloads.make_inputs(w)
+    Q, K, V = dev(inp.Q), dev(inp.K), dev(inp.V)
+    outs = [flare.forward(Q, K, V, want_stats=True) for _ in range(3)]
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+
+
+def test_encode_then_decode_equals_forward(oracle):
+    inp = workloads.make_inputs(workloads.CONFIGS["padded"].with_(B=2, N=700))
+    Q, K, V, mask = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask)
+    desc = flare.make_desc(Q, K)
+    Y1, Z1, le1, ld1 = flare.forward(Q, K, V, mask, want_stats=True)
+    ws = flare.alloc_workspace(desc, flare.OP_ENCODE)
+    Z2, le2 = torch.empty_like(Z1), torch.empty_like(le1)
+    flare.flare_encode(desc, Q, K, V, mask, Z2, le2, ws)
+    Y2, ld2 = torch.empty_like(Y1), torch.empty_like(ld1)
+    flare.flare_decode(desc, Q, K, Z2, Y2, ld2)
+    torch.cuda.synchronize()
+    assert torch.equal(Z1, Z2) and torch.equal(le1, le2) and torch.equal(Y1, Y2) and torch.equal(ld1, ld2)
+    # decode alone against the oracle's decode on the oracle's own Z
+    ref = oracle_forward(oracle, inp)
+    Zo = torch.from_numpy(ref["Z"]).float().cuda()
+    flare.flare_decode(desc, Q, K, Zo, Y2, None)
+    torch.cuda.synchronize()
+    assert rel_err(to_np64(Y2), ref["Y"]) <= TOL["bf16"]
+    # optional outputs may be NULL; Z may live in the workspace
+    wsf = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    Y3 = torch.empty_like(Y1)
+    flare.flare_forward(desc, Q, K, V, mask, Y3, None, None, None, wsf)
+    torch.cuda.synchronize()
+    assert torch.equal(Y1, Y3)
+
+
+def test_error_paths_on_device():
+    inp = workloads.make_random(1, 2, 64, 16, 16, dtype="bf16", seed=1)
+    Q, K, V = dev(inp.Q), dev(inp.K), dev(inp.V)
+    desc = flare.make_desc(Q, K)
+    Y = torch.empty_like(K)
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(flare.FlareError) as e:
+        flare.flare_forward(desc, Q, K, V, None, Y, None, None, None, small)
+    assert e.value.status == flare.ERR_WORKSPACE_TOO_SMALL
+    ws = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    import ctypes
+    lib = flare.load()
+    st = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    rc = lib.flare_forward(ctypes.byref(desc), Q.data_ptr(), K.data_ptr() + 2, V.data_ptr(), None, Y.data_ptr(), None,
+                           None, None, ws.data_ptr(), ws.numel(), st)
+    assert rc == flare.ERR_INVALID_ARG
+    rc = lib.flare_forward(ctypes.byref(desc), Q.data_ptr(), None, V.data_ptr(), None, Y.data_ptr(), None, None, None,
+                           ws.data_ptr(), ws.numel(), st)
+    assert rc == flare.ERR_INVALID_ARG
+    torch.cuda.synchronize()
