@@ -145,8 +145,12 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens per batch item in the oracle sample")
     ap.add_argument("--ref-tokens", type=int, default=16384)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--tokens", type=int, default=0, help="override N (a smaller case of the same workload)")
     args = ap.parse_args()
     w = get_workload(args.workload)
+    if args.tokens > 0:
+        w = w.with_(N=args.tokens, name=f"{w.name}@N={args.tokens}")
     if args.impl == "reference":
         return run_reference(args, w)
     if args.warmup < 3:
@@ -233,7 +237,20 @@ def main():
     ms_step = float(t.item()) / args.steps
     value = world * w.tokens / (ms_step / 1e3)
 
-    # end to end: pinned host buffers in, pinned host buffer out, through flare_forward_host
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V, mask, tensor_bytes, e)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist)
+
+
+def run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V, mask, tensor_bytes, e):
+    """End to end: pinned host buffers in, pinned host buffer out, through flare_forward_host."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     hQ, hK, hV = inp.Q.pin_memory(), inp.K.pin_memory(), inp.V.pin_memory()
     hmask = None if inp.key_mask is None else inp.key_mask.pin_memory()
     hY = torch.empty_like(inp.K).pin_memory()
@@ -252,14 +269,11 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     e2e_ms = float(t.item()) / args.e2e_steps
     h2d = 2 * tensor_bytes + w.H * w.M * w.D * e + (0 if mask is None else w.B * w.N)
-    e2e = {"value": world * w.tokens / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": tensor_bytes, "ms_per_step": e2e_ms}
+    return {"value": world * w.tokens / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": tensor_bytes, "ms_per_step": e2e_ms}
 
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
 
+def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist):
     peaks, peak_kind = load_peaks()
     # Roofline of the slower main kernel.  Per stage and head the contraction work is 4*N*M*D FLOP (scores and
     # value contraction); the bytes are K and V read (encode) or K read and Y written (decode), plus Q_lat.

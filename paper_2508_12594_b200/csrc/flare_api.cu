@@ -5,8 +5,11 @@
 #include <cstdio>
 #include <cstring>
 
+#include <cstdlib>
+
 #include "flare_common.cuh"
 #include "flare_simt.cuh"
+#include "flare_tc.cuh"
 
 using namespace flare;
 
@@ -90,7 +93,156 @@ SimtPlan simt_plan(const flare_desc_t *d, int sms) {
     return p;
 }
 
-int partials_for(const flare_desc_t *d, int sms) { return simt_plan(d, sms).P; }
+// The tensor-core kernels take bfloat16 with D in {16, 32, 64} and a positive scale; everything else (float32,
+// D = 8, non-positive scale) runs on the CUDA-core kernels.  FLARE_DEBUG_PATH=simt forces the latter.
+bool use_tc(const flare_desc_t *d) {
+    static const bool forced_simt = [] {
+        const char *e = std::getenv("FLARE_DEBUG_PATH");
+        return e != nullptr && std::strcmp(e, "simt") == 0;
+    }();
+    return !forced_simt && d->dtype == FLARE_DTYPE_BF16 && (d->D == 16 || d->D == 32 || d->D == 64) && d->scale > 0.f;
+}
+
+// Launch plan of the tensor-core encode: `pairs` CTAs per head along the latents (two 128-latent blocks each),
+// `splits` CTAs along N, about one CTA per SM in total.
+struct TcEncodePlan {
+    int tiles, pairs, splits, per_split, P;
+};
+
+TcEncodePlan tc_encode_plan(const flare_desc_t *d, int sms) {
+    TcEncodePlan p;
+    p.tiles = (d->N + kTile - 1) / kTile;
+    const int mb = (d->M + kTile - 1) / kTile;
+    p.pairs = (mb + 1) / 2;
+    long groups = (long)d->B * d->H * p.pairs;
+    long s = sms / groups;
+    if (s < 1) s = 1;
+    if (s > p.tiles) s = p.tiles;
+    p.splits = (int)s;
+    p.per_split = (mb == 1) ? 2 : 1;
+    p.P = p.splits * p.per_split;
+    return p;
+}
+
+int partials_for(const flare_desc_t *d, int sms) { return use_tc(d) ? tc_encode_plan(d, sms).P : simt_plan(d, sms).P; }
+
+// ---- TMA descriptors (the driver entry point is looked up at run time; the library does not link libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+CUtensorMapSwizzle swizzle_for(int D) {
+    return D == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : D == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+}
+
+// [B, N, H*D] bf16 viewed as a 3-D tensor (innermost H*D); box = one head's D columns x `rows` tokens.
+int make_token_map(CUtensorMap *m, const void *base, const flare_desc_t *d, int rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled not available");
+        return FLARE_ERR_CUDA;
+    }
+    const cuuint64_t C = (cuuint64_t)d->H * d->D;
+    cuuint64_t dims[3] = {C, (cuuint64_t)d->N, (cuuint64_t)d->B};
+    cuuint64_t strides[2] = {C * 2, C * 2 * (cuuint64_t)d->N};
+    cuuint32_t box[3] = {(cuuint32_t)d->D, (cuuint32_t)rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(d->D), CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled(tokens) failed: %d", (int)r);
+        return FLARE_ERR_CUDA;
+    }
+    return FLARE_OK;
+}
+
+// Q_lat [H*M, D] bf16 as a 2-D tensor; box = 16 latent rows.
+int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled not available");
+        return FLARE_ERR_CUDA;
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)d->D, (cuuint64_t)d->H * d->M};
+    cuuint64_t strides[1] = {(cuuint64_t)d->D * 2};
+    cuuint32_t box[2] = {(cuuint32_t)d->D, 16};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(d->D), CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled(latents) failed: %d", (int)r);
+        return FLARE_ERR_CUDA;
+    }
+    return FLARE_OK;
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D>
+int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
+                     const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st) {
+    CUtensorMap tmK, tmV, tmQ;
+    int rc;
+    if ((rc = make_token_map(&tmK, K, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmV, V, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
+    const size_t smem = EncodeSmem<D>::total();
+    static bool attr_set = false;
+    if (!attr_set) {
+        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    EncodeTcArgs a;
+    a.key_mask = mask; a.part_m = pm; a.part_l = pl; a.part_acc = pacc; a.status = status;
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.scale = d->scale; a.sl2 = d->scale * kLog2e;
+    a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
+    dim3 grid(p.splits, d->H * p.pairs, d->B);
+    encode_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+template <int D>
+int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                     float *lse_dec, uint32_t *status, cudaStream_t st) {
+    CUtensorMap tmK, tmQ;
+    int rc;
+    if ((rc = make_token_map(&tmK, K, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
+    const size_t smem = DecodeSmem<D>::total(d->M);
+    static bool attr_set = false;
+    if (!attr_set) {
+        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    DecodeTcArgs a;
+    a.Z = Z; a.Y = (__nv_bfloat16 *)Y; a.lse_dec = lse_dec; a.status = status;
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.sl2 = d->scale * kLog2e;
+    a.tiles = (d->N + kTile - 1) / kTile;
+    long per_head = sms / ((long)d->B * d->H);
+    if (per_head < 1) per_head = 1;
+    if (per_head > a.tiles) per_head = a.tiles;
+    dim3 grid((unsigned)per_head, d->H, d->B);
+    decode_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
 
 template <typename T>
 int launch_encode_simt(const flare_desc_t *d, const SimtPlan &p, const void *Q, const void *K, const void *V,
@@ -142,24 +294,40 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
                 float *lse_enc, void *ws, cudaStream_t st) {
     const DeviceInfo &di = device_info();
     const long rows = (long)d->B * d->H * d->M;
-    SimtPlan p = simt_plan(d, di.sms);
-    WorkspaceLayout w = make_layout(p.P, rows, d->D, false);
+    const int P = partials_for(d, di.sms);
+    WorkspaceLayout w = make_layout(P, rows, d->D, false);
     char *base = static_cast<char *>(ws);
     float *pm = reinterpret_cast<float *>(base + w.part_m);
     float *pl = reinterpret_cast<float *>(base + w.part_l);
     float *pacc = reinterpret_cast<float *>(base + w.part_acc);
     FLARE_CUDA(cudaMemsetAsync(base, 0, kHeaderBytes, st));
-    int rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)
+    int rc;
+    if (use_tc(d)) {
+        TcEncodePlan p = tc_encode_plan(d, di.sms);
+        uint32_t *status = reinterpret_cast<uint32_t *>(base);
+        rc = d->D == 16   ? launch_encode_tc<16>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+             : d->D == 32 ? launch_encode_tc<32>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+                          : launch_encode_tc<64>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
+    } else {
+        SimtPlan p = simt_plan(d, di.sms);
+        rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)
                                            : launch_encode_simt<__nv_bfloat16>(d, p, Q, K, V, mask, pm, pl, pacc, st);
+    }
     if (rc != FLARE_OK) return rc;
     const long total = rows * d->D;
-    merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(pm, pl, pacc, Z, lse_enc, p.P, rows, d->D);
+    merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(pm, pl, pacc, Z, lse_enc, P, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 
 int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
-                cudaStream_t st) {
+                uint32_t *status, cudaStream_t st) {
+    if (use_tc(d)) {
+        const int sms = device_info().sms;
+        return d->D == 16   ? launch_decode_tc<16>(d, sms, Q, K, Z, Y, lse_dec, status, st)
+               : d->D == 32 ? launch_decode_tc<32>(d, sms, Q, K, Z, Y, lse_dec, status, st)
+                            : launch_decode_tc<64>(d, sms, Q, K, Z, Y, lse_dec, status, st);
+    }
     return (d->dtype == FLARE_DTYPE_F32) ? launch_decode_simt<float>(d, Q, K, Z, Y, lse_dec, st)
                                          : launch_decode_simt<__nv_bfloat16>(d, Q, K, Z, Y, lse_dec, st);
 }
@@ -223,7 +391,7 @@ int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, con
     if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(Z) || !aligned16(Y) || (lse_dec && !aligned16(lse_dec)))
         return FLARE_ERR_INVALID_ARG;
     if ((rc = require_device()) != FLARE_OK) return rc;
-    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, (cudaStream_t)stream);
+    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, nullptr, (cudaStream_t)stream);
 }
 
 int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,
@@ -244,7 +412,7 @@ int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, co
     }
     rc = encode_impl(desc, Q_lat, K, V, key_mask, Z, lse_enc, workspace, (cudaStream_t)stream);
     if (rc != FLARE_OK) return rc;
-    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, (cudaStream_t)stream);
+    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, reinterpret_cast<uint32_t *>(workspace), (cudaStream_t)stream);
 }
 
 int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,

@@ -5,9 +5,28 @@
 // sums of the paper's design-principles appendix directly, with the usual running-maximum (online) softmax.
 #pragma once
 
+#include <type_traits>
+
 #include "flare_common.cuh"
 
 namespace flare {
+
+// Score q.k of one (latent, token) pair.  For float32 inputs the products are summed in double so that the
+// score, which is exponentiated, carries no float32 summation error; bfloat16 inputs sum in float.
+template <typename T, int D>
+__device__ __forceinline__ float score_dot(const float (&a)[D], const float *b) {
+    if constexpr (std::is_same<T, float>::value) {
+        double s = 0.0;
+#pragma unroll
+        for (int d = 0; d < D; ++d) s = fma((double)a[d], (double)b[d], s);
+        return (float)s;
+    } else {
+        float s = 0.f;
+#pragma unroll
+        for (int d = 0; d < D; ++d) s = fmaf(a[d], b[d], s);
+        return s;
+    }
+}
 
 constexpr int kSimtThreads = 256;
 constexpr int kSimtTileN = 32;  // tokens staged in shared memory per step
@@ -54,9 +73,7 @@ encode_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
             if (live) {
                 for (int j = g; j < kSimtTileN; j += G) {
                     if (!sValid[j]) continue;
-                    float s = 0.f;
-#pragma unroll
-                    for (int d = 0; d < D; ++d) s = fmaf(q[d], sK[j][d], s);
+                    const float s = score_dot<T, D>(q, sK[j]);
                     if (s > mx) {
                         float r = expf(mx - s);  // 0 on the first token (mx = -inf)
                         l *= r;
@@ -140,9 +157,7 @@ decode_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const float
         }
         __syncthreads();
         for (int j = 0; j < mc; ++j) {
-            float s = 0.f;
-#pragma unroll
-            for (int d = 0; d < D; ++d) s = fmaf(k[d], sQ[j][d], s);
+            const float s = score_dot<T, D>(k, sQ[j]);
             if (s > mx) {
                 float r = expf(mx - s);
                 l *= r;
