@@ -132,6 +132,31 @@ int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void 
                        void *workspace, size_t workspace_bytes, flare_stream_t stream);
 
 /*
+ * flare_encode without a caller-provided workspace.  (The paper has no counterpart: this exists for callers
+ * that are not allowed to allocate device memory at the point where they need the operator -- code running
+ * inside a memory-budgeted plugin or a real-time loop, hosts whose allocator is owned by another runtime and
+ * may not be re-entered, or late-bound callers that only hold the input and output tensors they were handed.)
+ *
+ * The per-split partial results go to a fixed array of FLARE_STATIC_SCRATCH_BYTES that is part of the
+ * library's device image: every GPU on which the library is loaded holds that much memory until the process
+ * exits, whether or not this function is ever called.  Nothing is allocated or freed by the call.
+ *
+ * Limits and rules:
+ *   - flare_workspace_bytes(desc, FLARE_OP_ENCODE) must not exceed FLARE_STATIC_SCRATCH_BYTES; a larger
+ *     problem is refused with FLARE_ERR_WORKSPACE_TOO_SMALL before any work is queued (flare_last_cuda_error()
+ *     then names both sizes).  Use flare_encode with your own workspace for those.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left; the function
+ *     clears the part that must start at zero itself.  Two calls whose GPU work overlaps in time (different
+ *     streams, or different host threads) race on it and produce garbage: serialise them.
+ *   - The first call on each device looks up the array's device address (with that device current) and caches
+ *     it.  Make that first call outside any stream capture.
+ * Arguments, outputs and status codes are otherwise those of flare_encode.
+ */
+#define FLARE_STATIC_SCRATCH_BYTES (8u << 20)
+int flare_encode_static_scratch(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
+                                const uint8_t *key_mask, float *Z, float *lse_enc, flare_stream_t stream);
+
+/*
  * After the stream has been synchronised: FLARE_OK, or FLARE_ERR_TIMEOUT if a kernel of the last call that
  * used `workspace` gave up on a bounded wait (its outputs are then undefined).  Reads one word from the
  * workspace with a blocking copy.

@@ -332,6 +332,29 @@ int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float
                                          : launch_decode_simt<__nv_bfloat16>(d, Q, K, Z, Y, lse_dec, st);
 }
 
+// Scratch of flare_encode_static_scratch: part of the device image, shared by every call on the device.
+// In host code this name is only a handle for cudaGetSymbolAddress; kernels must be given the looked-up address.
+static __device__ __align__(256) unsigned char g_static_scratch[FLARE_STATIC_SCRATCH_BYTES];
+void *g_static_scratch_addr[64] = {};
+
+// Device address of g_static_scratch on the current device (looked up once per device, then cached).
+int static_scratch_address(void **out) {
+    int dev = -1;
+    FLARE_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return FLARE_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void *p = nullptr;
+        FLARE_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (p == nullptr) {
+            snprintf(g_cuda_error, sizeof(g_cuda_error), "cudaGetSymbolAddress returned a null address");
+            return FLARE_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return FLARE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -381,6 +404,26 @@ int flare_encode(const flare_desc_t *desc, const void *Q_lat, const void *K, con
     if ((rc = require_device()) != FLARE_OK) return rc;
     if (workspace_bytes < flare_workspace_bytes(desc, FLARE_OP_ENCODE)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
     return encode_impl(desc, Q_lat, K, V, key_mask, Z, lse_enc, workspace, (cudaStream_t)stream);
+}
+
+int flare_encode_static_scratch(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
+                                const uint8_t *key_mask, float *Z, float *lse_enc, flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    if (!Q_lat || !K || !V || !Z) return FLARE_ERR_INVALID_ARG;
+    if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(V) || !aligned16(Z) || (lse_enc && !aligned16(lse_enc)))
+        return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    const size_t need = flare_workspace_bytes(desc, FLARE_OP_ENCODE);
+    if (need > (size_t)FLARE_STATIC_SCRATCH_BYTES) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "problem needs %zu bytes of scratch, the built-in array has %zu",
+                 need, (size_t)FLARE_STATIC_SCRATCH_BYTES);
+        return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    }
+    void *scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch)) != FLARE_OK) return rc;
+    // encode_impl zeroes the header words that must start at zero; every partial it later reads it first writes
+    return encode_impl(desc, Q_lat, K, V, key_mask, Z, lse_enc, scratch, (cudaStream_t)stream);
 }
 
 int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *Z, void *Y, float *lse_dec,

@@ -45,6 +45,7 @@ _SIGNATURES = {
     "flare_workspace_bytes": (_sz, [_dp, ctypes.c_int]),
     "flare_encode_partials": (ctypes.c_int, [_dp]),
     "flare_encode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "flare_encode_static_scratch": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "flare_decode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "flare_forward": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 14 + [_sz, _vp]),
@@ -142,6 +143,22 @@ def flare_encode(desc, Q, K, V, key_mask, Z, lse_enc, workspace, stream=None):
                              _ptr(Z, torch.float32, (B, H, M, D)), _ptr(lse_enc, torch.float32, (B, H, M)),
                              _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
     _raise(rc, "flare_encode")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def flare_encode_static_scratch(desc, Q, K, V, key_mask, Z, lse_enc, stream=None):
+    """flare_encode for callers that cannot allocate device memory: the partial results go to the library's
+    built-in scratch array (STATIC_SCRATCH_BYTES, shared by all calls on the device, so calls must not overlap
+    on the GPU).  Larger problems raise FlareError(ERR_WORKSPACE_TOO_SMALL)."""
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    rc = load().flare_encode_static_scratch(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, (B, N, H, D)),
+                                            _ptr(V, dt, (B, N, H, D)), _ptr(key_mask, torch.uint8, (B, N)),
+                                            _ptr(Z, torch.float32, (B, H, M, D)),
+                                            _ptr(lse_enc, torch.float32, (B, H, M)), _stream(stream))
+    _raise(rc, "flare_encode_static_scratch")
 
 
 def flare_decode(desc, Q, K, Z, Y, lse_dec, stream=None):
