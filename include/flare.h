@@ -114,7 +114,11 @@ int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, co
  *     dZ = W_dec^T dY;  dV = W_enc^T dZ;
  *     dS[m,n] = W_dec[n,m] (dY_n.Z_m - dY_n.Y_n) + W_enc[m,n] (dZ_m.V_n - dZ_m.Z_m);
  *     dQ_lat = scale * sum_b dS K;  dK = scale * dS^T Q_lat.
- * Z, lse_enc, lse_dec are the ones flare_forward wrote; Y is its output.
+ * Z, lse_enc, lse_dec are the ones flare_forward wrote; Y is its output (part of the saved set; the present
+ * kernels rebuild dY_n.Y_n = sum_m W_dec[n,m] (dY_n.Z_m) in float32 instead of reading the rounded Y, which
+ * is markedly more accurate where the latent rows a token mixes are nearly equal).
+ * dQ_lat, dK, dV are overwritten.  Workspace: flare_workspace_bytes(desc, FLARE_OP_BACKWARD) bytes holding dZ,
+ * per-split partial sums of dZ and dQ_lat, and one float per (b, n, h); nothing of size N x M.
  */
 int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
                    const uint8_t *key_mask, const void *Y, const void *dY, const float *Z, const float *lse_enc,

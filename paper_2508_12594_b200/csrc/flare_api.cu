@@ -9,6 +9,7 @@
 
 #include "flare_common.cuh"
 #include "flare_simt.cuh"
+#include "flare_bwd.cuh"
 #include "flare_tc.cuh"
 
 using namespace flare;
@@ -280,6 +281,88 @@ int launch_decode_simt(const flare_desc_t *d, const void *Q, const void *K, cons
     return FLARE_OK;
 }
 
+// Launch plans of the CUDA-core backward: pass A (dZ) reuses the encode plan; the dQ pass keeps three latent
+// rows per thread in shared memory and therefore caps its latent block at 64.
+SimtPlan bwd_dq_plan(const flare_desc_t *d, int sms) {
+    SimtPlan p = simt_plan(d, sms);
+    if (p.LM > 64) p.LM = 64;
+    p.G = kBwdThreads / p.LM;
+    p.P = p.splits * p.G;
+    return p;
+}
+
+struct BwdLayout {
+    size_t part, dz, de, dd, total;
+    int P;
+};
+
+BwdLayout bwd_layout(const flare_desc_t *d, int sms) {
+    BwdLayout w;
+    const long rows = (long)d->B * d->H * d->M;
+    const int pa = simt_plan(d, sms).P, pb = bwd_dq_plan(d, sms).P;
+    w.P = pa > pb ? pa : pb;
+    size_t off = kHeaderBytes;
+    w.part = off; off += align_up(sizeof(float) * (size_t)w.P * rows * d->D);
+    w.dz = off;   off += align_up(sizeof(float) * (size_t)rows * d->D);
+    w.de = off;   off += align_up(sizeof(float) * (size_t)rows);
+    w.dd = off;   off += align_up(sizeof(float) * (size_t)d->B * d->N * d->H);
+    w.total = off;
+    return w;
+}
+
+template <typename T, int D>
+int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V,
+                         const uint8_t *mask, const void *Y, const void *dY, const float *Z, const float *lse_enc,
+                         const float *lse_dec, float *dQ, void *dK, void *dV, char *ws, cudaStream_t st) {
+    const BwdLayout w = bwd_layout(d, sms);
+    float *part = reinterpret_cast<float *>(ws + w.part);
+    float *dZ = reinterpret_cast<float *>(ws + w.dz);
+    float *de = reinterpret_cast<float *>(ws + w.de);
+    float *dd = reinterpret_cast<float *>(ws + w.dd);
+    (void)Y;  // dY_n . Y_n is rebuilt from float32 quantities instead of the rounded stored Y
+    const long rows = (long)d->B * d->H * d->M;
+    const SimtPlan pa = simt_plan(d, sms), pb = bwd_dq_plan(d, sms);
+    FLARE_CUDA(cudaMemsetAsync(ws, 0, kHeaderBytes, st));
+    bwd_dz_simt_kernel<T, D><<<dim3(pa.splits, d->H, d->B), kBwdThreads, 0, st>>>(
+        (const T *)Q, (const T *)K, (const T *)dY, lse_dec, part, d->B, d->H, d->N, d->M, pa.LM, pa.chunk, d->scale);
+    FLARE_CUDA(cudaGetLastError());
+    bwd_dz_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(part, Z, dZ, de, pa.P, rows, d->D);
+    FLARE_CUDA(cudaGetLastError());
+    bwd_token_simt_kernel<T, D><<<dim3((d->N + 127) / 128, d->H, d->B), 128, 0, st>>>(
+        (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, lse_enc, lse_dec, (T *)dK, (T *)dV, dd,
+        d->B, d->H, d->N, d->M, d->scale);
+    FLARE_CUDA(cudaGetLastError());
+    const size_t dyn = sizeof(float) * 3 * (size_t)pb.LM * (D + 1);
+    static bool attr_set = false;
+    if (!attr_set) {
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(sizeof(float) * 3 * 64 * (D + 1))));
+        attr_set = true;
+    }
+    bwd_dq_simt_kernel<T, D><<<dim3(pb.splits, d->H, d->B), kBwdThreads, dyn, st>>>(
+        (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, dd, lse_enc, lse_dec, part, d->B, d->H,
+        d->N, d->M, pb.LM, pb.chunk, d->scale);
+    FLARE_CUDA(cudaGetLastError());
+    const long per_batch = (long)d->H * d->M * d->D;
+    bwd_dq_reduce_kernel<<<(unsigned)((per_batch + 255) / 256), 256, 0, st>>>(part, dQ, pb.P, d->B, d->H, d->M, d->D,
+                                                                             d->scale);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+template <typename T>
+int backward_simt(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const uint8_t *mask,
+                  const void *Y, const void *dY, const float *Z, const float *lse_enc, const float *lse_dec, float *dQ,
+                  void *dK, void *dV, char *ws, cudaStream_t st) {
+    switch (d->D) {
+        case 8: return launch_backward_simt<T, 8>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
+        case 16: return launch_backward_simt<T, 16>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
+        case 32: return launch_backward_simt<T, 32>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
+        case 64: return launch_backward_simt<T, 64>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
+        default: return FLARE_ERR_UNSUPPORTED;
+    }
+}
+
 int require_device() {
     const DeviceInfo &di = device_info();
     if (di.checked == -2) {
@@ -388,7 +471,7 @@ size_t flare_workspace_bytes(const flare_desc_t *desc, int op) {
         case FLARE_OP_ENCODE: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, false).total;
         case FLARE_OP_DECODE: return kHeaderBytes;
         case FLARE_OP_FORWARD: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, true).total;
-        case FLARE_OP_BACKWARD: return 0;
+        case FLARE_OP_BACKWARD: return bwd_layout(desc, device_info().sms).total;
         default: return 0;
     }
 }
@@ -462,11 +545,20 @@ int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, c
                    const void *Y, const void *dY, const float *Z, const float *lse_enc, const float *lse_dec,
                    float *dQ_lat, void *dK, void *dV, void *workspace, size_t workspace_bytes,
                    flare_stream_t stream) {
-    (void)Q_lat; (void)K; (void)V; (void)key_mask; (void)Y; (void)dY; (void)Z; (void)lse_enc; (void)lse_dec;
-    (void)dQ_lat; (void)dK; (void)dV; (void)workspace; (void)workspace_bytes; (void)stream;
     int rc = check_desc(desc);
     if (rc != FLARE_OK) return rc;
-    return FLARE_ERR_UNSUPPORTED;
+    const void *ptrs[] = {Q_lat, K, V, Y, dY, Z, lse_enc, lse_dec, dQ_lat, dK, dV, workspace};
+    for (const void *p : ptrs)
+        if (p == nullptr || !aligned16(p)) return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    if (workspace_bytes < flare_workspace_bytes(desc, FLARE_OP_BACKWARD)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    const int sms = device_info().sms;
+    char *ws = static_cast<char *>(workspace);
+    cudaStream_t st = (cudaStream_t)stream;
+    return desc->dtype == FLARE_DTYPE_F32
+               ? backward_simt<float>(desc, sms, Q_lat, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ_lat, dK, dV, ws, st)
+               : backward_simt<__nv_bfloat16>(desc, sms, Q_lat, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ_lat, dK,
+                                              dV, ws, st);
 }
 
 int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void *hK, const void *hV,

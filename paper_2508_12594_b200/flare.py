@@ -48,7 +48,7 @@ _SIGNATURES = {
     "flare_encode_static_scratch": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "flare_decode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "flare_forward": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
-    "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 14 + [_sz, _vp]),
+    "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 13 + [_sz, _vp]),
     "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
     "flare_check": (ctypes.c_int, [_vp, _vp]),
 }
@@ -222,3 +222,15 @@ def forward(Q, K, V, key_mask=None, scale=1.0, want_stats=False, stream=None):
     ld = torch.empty(B, N, H, dtype=torch.float32, device=K.device)
     flare_forward(desc, Q, K, V, key_mask, Y, Z, le, ld, ws, stream)
     return (Y, Z, le, ld) if want_stats else Y
+
+
+def forward_backward(Q, K, V, dY, key_mask=None, scale=1.0, stream=None):
+    """Convenience: flare_forward (keeping Z and the log-sum-exp rows) then flare_backward.
+    Returns (Y, dQ_lat [H,M,D] float32, dK, dV)."""
+    desc = make_desc(Q, K, scale)
+    Y, Z, le, ld = forward(Q, K, V, key_mask, scale, want_stats=True, stream=stream)
+    ws = alloc_workspace(desc, OP_BACKWARD, K.device)
+    dQ = torch.empty(desc.H, desc.M, desc.D, dtype=torch.float32, device=K.device)
+    dK, dV = torch.empty_like(K), torch.empty_like(V)
+    flare_backward(desc, Q, K, V, key_mask, Y, dY, Z, le, ld, dQ, dK, dV, ws, stream)
+    return Y, dQ, dK, dV

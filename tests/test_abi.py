@@ -31,6 +31,17 @@ def test_every_declared_symbol_is_exported(lib):
     assert sorted(flare.exported_symbols()) == names
 
 
+def test_binding_argument_counts_match_the_header():
+    """Every prototype in the header has as many parameters as the binding's ctypes signature."""
+    text = open(os.path.join(ROOT, "include", "flare.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    protos = dict(re.findall(r"\b(flare_[a-z_]+)\s*\(([^)]*)\)\s*;", text))
+    assert set(protos) == set(flare._SIGNATURES)
+    for name, params in protos.items():
+        n = 0 if params.strip() in ("", "void") else params.count(",") + 1
+        assert n == len(flare._SIGNATURES[name][1]), name
+
+
 def test_status_strings(lib):
     assert lib.flare_status_string(0) == b"ok"
     for s in range(1, 7):

@@ -1,0 +1,137 @@
+"""Parity of flare_backward against the CPU oracle's gradients, element by element, through the C-ABI (needs a B200).
+
+The gradients are those of sum(Y * dY).  Tolerance per tensor (dQ_lat, dK, dV):
+    |got - ref| <= tol * RMS(ref) + store_ulp * |ref|     element by element,
+tol = 2e-2 for bfloat16 inputs (the forward's bound) and 1e-4 for float32 (a gradient entry is a sum of M or N
+signed terms dS * q, each carrying the float32 rounding of an exponential and of two D-term dot products that
+nearly cancel, dY.Z_m - dY.Y, so its error relative to the tensor's RMS is a few 1e-6 and grows with sqrt(M)).
+store_ulp = 2^-8 for dK and dV stored as bfloat16, 0 otherwise: gradients are heavy-tailed (max/RMS of 20 to 60
+on these workloads, against 3 to 4 for Y), so rounding the exact value of the largest entries to bfloat16 alone
+is an error of 6e-2 to 9e-2 * RMS; the second term allows exactly that one rounding and nothing more.
+The backward forms dY_n . Y_n from float32 quantities, not from the stored bfloat16 Y: with the stored Y, the one
+rounding of Y alone moved dK and dQ by up to 7e-2 * RMS on these workloads (measured), because it does not cancel
+in dS where the latent rows a token mixes are nearly equal.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2508_12594_b200 import flare, workloads
+from tests._util import dev, rel_err, to_np64
+
+pytestmark = pytest.mark.gpu
+
+GRAD_TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+def gpu_backward(inp, scale=1.0):
+    Q, K, V, mask, dY = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask), dev(inp.dY)
+    Y, dQ, dK, dV = flare.forward_backward(Q, K, V, dY, mask, scale)
+    torch.cuda.synchronize()
+    return dict(dQ=to_np64(dQ), dK=to_np64(dK), dV=to_np64(dV))
+
+
+def oracle_backward(oracle, inp, scale=1.0):
+    mask = None if inp.key_mask is None else inp.key_mask.numpy()
+    return oracle.backward(to_np64(inp.Q), to_np64(inp.K), to_np64(inp.V), to_np64(inp.dY), key_mask=mask, scale=scale)
+
+
+def assert_grads_close(got, ref, dtype, what, floor=None):
+    """`floor`: optional dict of lower bounds on the RMS used as the error scale (for exactly-zero gradients)."""
+    for name in ("dV", "dK", "dQ"):
+        rms = float(np.sqrt(np.mean(ref[name] ** 2)))
+        if floor is not None:
+            rms = max(rms, floor[name])
+        store_ulp = 2.0 ** -8 if (dtype == "bf16" and name != "dQ") else 0.0
+        excess = np.abs(got[name] - ref[name]) - store_ulp * np.abs(ref[name])
+        e = float(excess.max()) / max(rms, 1e-300)
+        assert e <= GRAD_TOL[dtype], f"{what} {name}: (max|err| - ulp)/RMS = {e:.3e} > {GRAD_TOL[dtype]}"
+
+
+CASES = [
+    workloads.CONFIGS["tiny"].with_(backward=True),
+    workloads.CONFIGS["padded"].with_(B=3, N=1000),
+    workloads.sweep_point(2500, 32),
+    workloads.sweep_point(1300, 128),
+    workloads.sweep_point(700, 512),
+    workloads.CONFIGS["mesh2d"].with_(B=2, N=1501, backward=True),
+]
+
+
+@pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
+@pytest.mark.parametrize("paper_scale", [True, False], ids=["s=1", "s=1/sqrtD"])
+def test_backward_scaled_down_workloads(oracle, w, paper_scale):
+    scale = 1.0 if paper_scale else w.D ** -0.5
+    inp = workloads.make_inputs(w)
+    assert_grads_close(gpu_backward(inp, scale), oracle_backward(oracle, inp, scale), w.dtype, w.name)
+
+
+EDGE = [
+    # B, H, N, M, D, dtype, masked_fraction
+    (1, 1, 1, 1, 8, "f32", 0.0),
+    (2, 3, 7, 16, 8, "bf16", 0.0),
+    (1, 2, 129, 64, 32, "bf16", 0.3),
+    (2, 1, 300, 256, 64, "bf16", 0.0),
+    (1, 1, 515, 512, 16, "bf16", 0.5),
+    (3, 2, 333, 5, 32, "f32", 0.4),
+    (1, 1, 600, 300, 64, "f32", 0.0),
+    (1, 4, 64, 1, 16, "f32", 0.0),
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=lambda c: "B{}H{}N{}M{}D{}{}m{}".format(*c))
+def test_backward_edge_shapes(oracle, case):
+    B, H, N, M, D, dtype, mf = case
+    inp = workloads.make_random(B, H, N, M, D, dtype=dtype, seed=N + M, masked_fraction=mf, with_dy=True, k_std=0.8)
+    assert_grads_close(gpu_backward(inp), oracle_backward(oracle, inp), dtype, str(case))
+
+
+def test_backward_single_token(oracle):
+    """N = 1: Z_m = V_0 and Y_0 = V_0 whatever the scores, so dK = dQ = 0 and dV_0 = dY_0.  The exact zeros are
+    compared on the scale of the terms that cancel, |dY| |V| |Q|."""
+    inp = workloads.make_random(1, 1, 1, 16, 16, dtype="bf16", seed=17, with_dy=True, k_std=0.8)
+    got, ref = gpu_backward(inp), oracle_backward(oracle, inp)
+    np.testing.assert_allclose(ref["dV"], to_np64(inp.dY), rtol=1e-12)
+    scale = float(inp.dY.double().abs().max() * inp.V.double().abs().max() * inp.Q.double().abs().max())
+    assert_grads_close(got, ref, "bf16", "N=1", floor=dict(dV=0.0, dK=scale, dQ=scale))
+
+
+def test_backward_masked_tokens_and_empty_items(oracle):
+    """Masked tokens get dV = 0 exactly; an item with no valid token gets dV = 0 and dK from the decode term only."""
+    inp = workloads.make_random(2, 2, 200, 16, 16, dtype="f32", seed=5, with_dy=True)
+    mask = (torch.rand(2, 200, generator=torch.Generator().manual_seed(1)) > 0.3).to(torch.uint8)
+    mask[1] = 0
+    inp.key_mask = mask
+    got, ref = gpu_backward(inp), oracle_backward(oracle, inp)
+    assert_grads_close(got, ref, "f32", "masked")
+    assert (got["dV"][mask.numpy() == 0] == 0).all()
+
+
+def test_backward_bitwise_reproducible():
+    inp = workloads.make_inputs(workloads.CONFIGS["padded"].with_(B=2, N=3000))
+    Q, K, V, mask, dY = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask), dev(inp.dY)
+    outs = [flare.forward_backward(Q, K, V, dY, mask) for _ in range(3)]
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+
+
+def test_backward_error_paths():
+    inp = workloads.make_random(1, 2, 64, 16, 16, dtype="bf16", seed=1, with_dy=True)
+    Q, K, V, dY = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.dY)
+    desc = flare.make_desc(Q, K)
+    Y, Z, le, ld = flare.forward(Q, K, V, want_stats=True)
+    dQ = torch.empty(2, 16, 16, dtype=torch.float32, device="cuda")
+    dK, dV = torch.empty_like(K), torch.empty_like(V)
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(flare.FlareError) as e:
+        flare.flare_backward(desc, Q, K, V, None, Y, dY, Z, le, ld, dQ, dK, dV, small)
+    assert e.value.status == flare.ERR_WORKSPACE_TOO_SMALL
+    ws = flare.alloc_workspace(desc, flare.OP_BACKWARD)
+    import ctypes
+    rc = flare.load().flare_backward(ctypes.byref(desc), Q.data_ptr(), K.data_ptr(), V.data_ptr(), None, Y.data_ptr(),
+                                     dY.data_ptr(), Z.data_ptr(), None, ld.data_ptr(), dQ.data_ptr(), dK.data_ptr(),
+                                     dV.data_ptr(), ws.data_ptr(), ws.numel(), None)
+    assert rc == flare.ERR_INVALID_ARG
+    torch.cuda.synchronize()
