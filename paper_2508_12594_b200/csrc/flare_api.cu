@@ -120,7 +120,7 @@ TcEncodePlan tc_encode_plan(const flare_desc_t *d, int sms) {
     if (s < 1) s = 1;
     if (s > p.tiles) s = p.tiles;
     p.splits = (int)s;
-    p.per_split = (mb == 1) ? 2 : 1;
+    p.per_split = (mb == 1) ? 4 : 2;
     p.P = p.splits * p.per_split;
     return p;
 }
@@ -236,6 +236,8 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
     a.sl2 = d->scale * kLog2e;
     a.tiles = (d->N + kTile - 1) / kTile;
+    a.plan = make_decode_plan(d->M, D);
+    if (a.plan.cs == 0) return FLARE_ERR_UNSUPPORTED;
     long per_head = sms / ((long)d->B * d->H);
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;

@@ -5,9 +5,17 @@
 //   decode  S = K_tile Q_h^T   (tokens on the 128 TMEM lanes, latents on columns)   Y    = P Z_h
 // Scores land in tensor memory; one thread owns one lane (one latent in encode, one token in decode), so row
 // maxima and sums need no shuffles.  The bf16 weights P are written back over the scores in tensor memory and
-// feed the second contraction as its A operand.  Warp roles: warp 0 issues TMA loads, warp 1 issues the MMAs
-// and owns the TMEM allocation, warps 4-7 and 8-11 are two softmax groups that alternate on two TMEM buffers
-// so that one group's exponentials overlap the other's MMAs.
+// feed the second contraction as its A operand.
+//
+// Two resources limit both kernels, and neither is the one a roofline of FLOPs and bytes names.  Every
+// (latent, token) pair needs one exponential on the special-function unit (16 per clock per SM), and every
+// tcgen05.mma of this shape (M = 128, K = 16) holds the tensor pipe for about 107 cycles whatever its N
+// (measured), so the value contraction costs one such slot per 16 latents (decode) or tokens (encode): about
+// as long as the exponentials of the same block.  The CTA is built to keep both busy at once: warp 0 issues
+// TMA loads, warp 1 issues the MMAs and owns the TMEM allocation, and sixteen softmax warps (four per
+// scheduler) form four groups of four warps.  A group owns one TMEM score buffer, or a range of columns of a
+// shared one, with its own running maximum, sum and accumulator columns; while one group waits for its MMAs
+// the other three keep the schedulers fed.
 #pragma once
 
 #include "flare_common.cuh"
@@ -15,7 +23,9 @@
 
 namespace flare {
 
-constexpr int kTcThreads = 384;
+constexpr int kSoftmaxGroups = 4;                            // groups of 4 warps (128 threads = 128 TMEM lanes)
+constexpr int kFirstSoftmaxWarp = 2;
+constexpr int kTcThreads = (kFirstSoftmaxWarp + 4 * kSoftmaxGroups) * 32;  // 576
 constexpr int kTile = 128;       // tokens per tile (decode: TMEM lanes; encode: score columns)
 constexpr int kDecStages = 4;    // K tiles in flight (decode)
 constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode)
@@ -41,6 +51,102 @@ struct TileGeom {
     __device__ static __forceinline__ int swz(int r) { return RB == 32 ? ((r >> 2) & 1) : RB == 64 ? ((r >> 1) & 3) : (r & 7); }
 };
 
+// ------------------------------------------------------------------------------------- softmax arithmetic
+// Row maximum over NV (16 or 32) float32 scores held as raw bits.
+template <int NV>
+__device__ __forceinline__ float max_of(const uint32_t *r, float m) {
+#pragma unroll
+    for (int k = 0; k < NV; k += 2) m = ptx::max3(m, __uint_as_float(r[k]), __uint_as_float(r[k + 1]));
+    return m;
+}
+
+// p = 2^(s * sl2 + neg) for NV scores; bf16 pairs to pk, float32 sums into sum2 (two interleaved partial sums).
+// With kMasked, scores whose bit in `valid` is clear (or all of them if `dead`) get weight exactly 0.
+template <int NV, bool kMasked>
+__device__ __forceinline__ void exp_chunk(const uint32_t *r, uint32_t *pk, float2 sl2p, float2 negp, float2 &sum2,
+                                          uint32_t valid = 0xffffffffu, bool dead = false) {
+#pragma unroll
+    for (int k = 0; k < NV / 2; ++k) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * k]), __uint_as_float(r[2 * k + 1])), sl2p, negp);
+        float2 p = make_float2(ptx::ex2(x.x), ptx::ex2(x.y));
+        if (kMasked) {
+            if (dead || !((valid >> (2 * k)) & 1)) p.x = 0.f;
+            if (dead || !((valid >> (2 * k + 1)) & 1)) p.y = 0.f;
+        }
+        sum2 = __fadd2_rn(sum2, p);
+        pk[k] = ptx::pack_bf16(p.x, p.y);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ decode
+// How the four softmax groups share tensor memory in decode.  `cs` groups split the M score columns of one
+// buffer into ranges of `part_w` columns (the last may be shorter); `nbuf` buffers of `cb` columns hold
+// different token tiles.  The Y accumulator of a column range sits in columns of that range that its packed
+// bf16 weights leave free (`alias`), else after the scores.  Every range is a pipeline of its own: its scores
+// come from their own MMA, its weights go to the value contraction a few columns at a time as they are written
+// (so that the tensor pipe works on one part of the row while the exponentials of the next are evaluated), and
+// the ranges of a tile meet again only when its rows of Y are written.
+//
+// Z enters the value contraction as two bf16 halves (hi = round(z), lo = round(z - hi), about 16 mantissa
+// bits: with plain bf16 rows the rounding of Z alone reaches the error bound where max|Z| is several times
+// RMS(Y)).  With a narrow head the halves sit side by side as one B operand of width 2D, so that the split
+// costs no extra MMA ([P Z_hi | P Z_lo], added when Y is written).
+struct DecodePlan {
+    int cs, nbuf, part_w, alias, cb, ncols;
+};
+
+// Columns of one Y accumulator.
+__host__ __device__ constexpr int decode_y_cols(int D) { return D <= 32 ? 2 * D : D; }
+
+// Column choreography of one range of `len` score columns with aliasing.  The softmax walks the scores from the
+// top column down in chunks of 32; a chunk's columns are free once read.  With a Y accumulator of `yc` columns,
+// the first yc/16 chunks free 2*yc columns, which take those chunks' packed weights (16 columns each, top
+// down) and, below them, Y; every later chunk's weights go to the bottom half of the chunk's own columns.
+__host__ __device__ inline int decode_y_alias_col(int len, int yc) { return len - 2 * yc; }
+// First column (within the range) of the packed weights of the chunk whose scores start at column `lo`.
+__host__ __device__ inline int decode_p_col(int len, int yc, int lo, bool alias) {
+    const int k = (len - 1 - lo) / 32;                         // chunk index counted from the top
+    return (alias && k < yc / 16) ? len - 16 * (k + 1) : lo;
+}
+// Score columns per hand-over of weights to the value contraction: at most four per range and tile, and the
+// first covers the 2*yc columns that make room for Y.
+__host__ __device__ inline int decode_handover_cols(int len, int yc) {
+    int u = ((len + 3) / 4 + 31) & ~31;
+    if (u < 2 * yc) u = 2 * yc;
+    return u < 32 ? 32 : u;
+}
+
+__host__ __device__ inline int decode_part_len(const DecodePlan &p, int M, int c) {
+    const int start = c * p.part_w;
+    const int len = M - start < p.part_w ? M - start : p.part_w;
+    return len > 0 ? len : 0;
+}
+
+inline DecodePlan make_decode_plan(int M, int D) {
+    const int yc = decode_y_cols(D);
+    DecodePlan best{};
+    int best_groups = 0;
+    for (int cs = 1; cs <= 4; cs *= 2) {
+        DecodePlan p;
+        p.cs = cs;
+        p.part_w = ((M / 16 + cs - 1) / cs) * 16;
+        if ((cs - 1) * p.part_w >= M) continue;                 // an empty column range
+        p.alias = 1;
+        for (int c = 0; c < cs; ++c)
+            if (decode_part_len(p, M, c) < 2 * yc) p.alias = 0;
+        p.cb = ((p.alias ? M : M + cs * yc) + 31) & ~31;
+        if (p.cb > 512) continue;
+        p.nbuf = 512 / p.cb < kSoftmaxGroups / cs ? 512 / p.cb : kSoftmaxGroups / cs;
+        p.ncols = 32;
+        while (p.ncols < p.nbuf * p.cb) p.ncols *= 2;
+        if (p.nbuf * cs > best_groups) {
+            best_groups = p.nbuf * cs;
+            best = p;
+        }
+    }
+    return best;
+}
+
 struct DecodeTcArgs {
     const float *Z;      // [B,H,M,D]
     __nv_bfloat16 *Y;    // [B,N,H,D]
@@ -49,6 +155,7 @@ struct DecodeTcArgs {
     int B, H, N, M;
     float sl2;           // scale * log2(e)
     int tiles;           // ceil(N / 128)
+    DecodePlan plan;
 };
 
 // Shared-memory carve-up of the decode kernel.
@@ -56,15 +163,21 @@ template <int D>
 struct DecodeSmem {
     using G = TileGeom<D>;
     static constexpr size_t k_off = 0;
-    // K tiles in flight: kDecStages, or 2 when Q_h and the two halves of Z_bh leave no room for more
+    static constexpr size_t kBarBytes = 512;
+    static constexpr size_t kTail = kBarBytes + 2 * kSoftmaxGroups * kTile * sizeof(float);  // barriers + row statistics
+    // K tiles in flight: as many of kDecStages as fit beside Q_h and the two halves of Z_bh.  (A K tile is free
+    // again as soon as its score MMAs have run, so even one stage leaves a whole tile's softmax to hide the load.)
     __host__ __device__ static int stages(int M) {
-        return ((size_t)kDecStages * G::TILE_BYTES + (size_t)3 * M * G::RB + 2304 <= 227 * 1024) ? kDecStages : 2;
+        int s = kDecStages;
+        while (s > 1 && (size_t)s * G::TILE_BYTES + (size_t)3 * M * G::RB + kTail + 2048 > 227 * 1024) --s;
+        return s;
     }
     __host__ __device__ static size_t q_off(int M) { return (size_t)stages(M) * G::TILE_BYTES; }
     __host__ __device__ static size_t z_off(int M) { return q_off(M) + (size_t)M * G::RB; }  // [hi | lo], M rows each
     __host__ __device__ static size_t bar_off(int M) { return align_up(z_off(M) + (size_t)2 * M * G::RB, 1024); }
+    __host__ __device__ static size_t stat_off(int M) { return bar_off(M) + kBarBytes; }
     __host__ __device__ static size_t total(int M) {
-        size_t t = bar_off(M) + 256 + 1024;  // barriers and flags, plus slack to align the base to 1024
+        size_t t = bar_off(M) + kTail + 1024;  // plus slack to align the base to 1024
         return t < kTcMinSmem ? kTcMinSmem : t;
     }
 };
@@ -84,9 +197,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint8_t *sZ = smem + SM::z_off(M);
     const int nstages = SM::stages(M);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off(M));
-    // barrier indices
-    enum { K_FULL = 0, K_EMPTY = K_FULL + kDecStages, S_FULL = K_EMPTY + kDecStages, P_FULL = S_FULL + 2,
-           Y_FULL = P_FULL + 2, BUF_EMPTY = Y_FULL + 2, Q_FULL = BUF_EMPTY + 2, NBARS };
+    float *stat_m = reinterpret_cast<float *>(smem + SM::stat_off(M));   // [group][128] row maxima (log2 units)
+    float *stat_l = stat_m + kSoftmaxGroups * kTile;                      // [group][128] row sums
+    constexpr int NG = kSoftmaxGroups;
+    // S_FULL, Y_FULL: one per group (column range of a buffer); P_CHUNK: four hand-overs per group; BUF_EMPTY: per buffer
+    enum { K_FULL = 0, K_EMPTY = K_FULL + kDecStages, S_FULL = K_EMPTY + kDecStages, P_CHUNK = S_FULL + NG,
+           Y_FULL = P_CHUNK + 4 * NG, BUF_EMPTY = Y_FULL + NG, Q_FULL = BUF_EMPTY + NG, NBARS };
+    static_assert(NBARS * 8 + 8 <= SM::kBarBytes, "barrier area too small");
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -96,31 +213,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int t_end = (int)((long)a.tiles * (blockIdx.x + 1) / gridDim.x);
     const int ntiles = t_end - t_begin;
 
-    // TMEM plan: per buffer S occupies M columns, P (bf16 pairs) overlays columns [0, M/2), Y sits after P
-    // when that still fits inside the S columns, otherwise after S.
-    const int nbuf = (M <= 256) ? 2 : 1;
-    const int p_end = (M / 2 + 15) & ~15;
-    const int y_off = (p_end + D <= M) ? p_end : M;
-    const int cb = (((y_off + D > M) ? y_off + D : M) + 31) & ~31;  // columns per buffer
-    uint32_t ncols = 32;
-    while ((int)ncols < nbuf * cb) ncols *= 2;
+    const DecodePlan pl = a.plan;
+    const int cs = pl.cs, nbuf = pl.nbuf, cb = pl.cb;
+    constexpr int YC = decode_y_cols(D);
+    constexpr bool kWide = YC == 2 * D;                         // one MMA over [Z_hi | Z_lo] (N = 2D) per 16 latents
+    // column of the Y accumulator of range c, relative to its buffer
+    auto y_col = [&](int c) {
+        if (!pl.alias) return M + c * YC;
+        return c * pl.part_w + decode_y_alias_col(decode_part_len(pl, M, c), YC);
+    };
 
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBARS; ++i) {
-            uint32_t count = (i >= P_FULL && i < P_FULL + 2) || (i >= BUF_EMPTY && i < BUF_EMPTY + 2) ? 128u : 1u;
-            ptx::mbar_init(bar(i), count);
+            const bool counted = (i >= P_CHUNK && i < P_CHUNK + 4 * NG) || (i >= BUF_EMPTY && i < BUF_EMPTY + NG);
+            ptx::mbar_init(bar(i), counted ? 128u : 1u);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
         ptx::prefetch_tensormap(&tmQ);
     }
-    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), ncols);
-    // Z_bh -> two bf16 halves (hi = round(z), lo = round(z - hi)) so that the latent sequence enters the second
-    // contraction with about 16 mantissa bits; rows of RB bytes in the swizzled layout the MMA's B operand
-    // expects (latent-major rows).
+    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), (uint32_t)pl.ncols);
+    // Z_bh -> two bf16 halves (hi = round(z), lo = round(z - hi)); rows of RB bytes in the swizzled layout the
+    // MMA's B operand expects (latent-major rows), the lo half M rows after the hi half.
     {
         const float *Zg = a.Z + ((size_t)b * a.H + h) * M * D;
         for (int i = threadIdx.x; i < M * (D / 8); i += kTcThreads) {
@@ -163,110 +280,231 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const int nsplit = (M + 255) / 256;                 // score MMAs per k-step (N <= 256 each)
-            const uint32_t idescS0 = ptx::instr_desc_bf16(128, M < 256 ? M : 256, 0, 0);
-            const uint32_t idescS1 = ptx::instr_desc_bf16(128, M > 256 ? M - 256 : 16, 0, 0);
-            const uint32_t idescY = ptx::instr_desc_bf16(128, D, 0, 1);
-            const uint32_t qaddr = ptx::smem_u32(sQ), zaddr = ptx::smem_u32(sZ);
+            // The MMA thread is a scheduler over the groups' pipelines: for each group it issues, whichever is
+            // ready, the scores of the group's next tile (K tile landed, buffer drained) or the value contraction of
+            // the next columns of weights the group has handed over.
+            const uint32_t idescY = ptx::instr_desc_bf16(128, YC, 0, 1);
+            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ);
+            // Z as the MN-major B operand: 8-row groups SBO apart; in the wide form the lo half is the second block
+            // along N, M rows further on.  Descriptor address fields are in 16-byte units.
+            const uint64_t zdesc = ptx::smem_desc(ptx::smem_u32(sZ), kWide ? (uint32_t)(M * G::RB) : (uint32_t)G::SBO,
+                                                  G::SBO, G::SWZ);
+            const int ng = nbuf * cs;
+            int len_g[NG], ycol_g[NG], ho_g[NG];                // per group: range length, Y column, columns per hand-over
+            int s_next[NG], v_next[NG], v_top[NG];              // per group: tiles whose scores / values are issued; columns left
+            int s_count[NG];                                    // per buffer: ranges of the current tile whose scores are issued
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
+                const int c = g % cs;
+                len_g[g] = g < ng ? decode_part_len(pl, M, c) : 0;
+                ycol_g[g] = g < ng ? y_col(c) : 0;
+                ho_g[g] = decode_handover_cols(len_g[g], YC);
+                s_next[g] = v_next[g] = v_top[g] = s_count[g] = 0;
+            }
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrDecode | 2);
-            auto issue_scores = [&](int i) -> bool {
-                const int s = i % nstages, j = i % nbuf, u = i / nbuf;
-                if (!ptx::mbar_wait(bar(K_FULL + s), (i / nstages) & 1, abort_flag, kErrDecode | 3)) return false;
-                if (!ptx::mbar_wait(bar(BUF_EMPTY + j), (u & 1) ^ 1, abort_flag, kErrDecode | 4)) return false;
-                ptx::tc_fence_after();
-                const uint32_t kaddr = ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES);
-                for (int ns = 0; ns < nsplit; ++ns)
-                    for (int k = 0; k < D / 16; ++k)
-                        ptx::mma_ss(tm + j * cb + ns * 256, ptx::smem_desc(kaddr + k * 32, 16, G::SBO, G::SWZ),
-                                    ptx::smem_desc(qaddr + ns * 256 * G::RB + k * 32, 16, G::SBO, G::SWZ),
-                                    ns == 0 ? idescS0 : idescS1, k > 0);
-                ptx::mma_commit(bar(S_FULL + j));
-                ptx::mma_commit(bar(K_EMPTY + s));
-                return true;
-            };
-            auto issue_values = [&](int i) -> bool {
-                const int j = i % nbuf, u = i / nbuf;
-                if (!ptx::mbar_wait(bar(P_FULL + j), u & 1, abort_flag, kErrDecode | 5)) return false;
-                ptx::tc_fence_after();
-                for (int half = 0; half < 2; ++half)            // Y = P Z_hi + P Z_lo
-                    for (int k = 0; k < M / 16; ++k)
-                        ptx::mma_ts(tm + j * cb + y_off, tm + j * cb + k * 8,
-                                    ptx::smem_desc(zaddr + (half * M + k * 16) * G::RB, G::SBO, G::SBO, G::SWZ), idescY,
-                                    half > 0 || k > 0);
-                ptx::mma_commit(bar(Y_FULL + j));
-                return true;
-            };
-            for (int i = 0; ok && i < ntiles; ++i) {
-                ok = issue_scores(i);
-                if (nbuf == 2) {
-                    if (ok && i > 0) ok = issue_values(i - 1);
-                } else if (ok) {
-                    ok = issue_values(i);
+            int remaining = 0;                                  // (group, tile) pairs still to finish
+            for (int g = 0; g < ng; ++g) remaining += (ntiles - g / cs + nbuf - 1) / nbuf;
+            uint64_t t0 = 0;                                    // start of the current stretch without progress
+            uint32_t spins = 0;
+            while (ok && remaining > 0) {
+                bool progressed = false;
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                    if (g >= ng) break;
+                    const int j = g / cs, c = g % cs;
+                    const uint32_t buf = tm + j * cb;
+                    if (s_next[g] == v_next[g]) {               // idle: try to issue the scores of the group's next tile
+                        const int u = s_next[g], i = j + u * nbuf;
+                        if (i >= ntiles) continue;
+                        const int s = i % nstages;
+                        if (!ptx::mbar_test(bar(K_FULL + s), (i / nstages) & 1) ||
+                            !ptx::mbar_test(bar(BUF_EMPTY + j), (u & 1) ^ 1))
+                            continue;
+                        ptx::tc_fence_after();
+                        const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), 16, G::SBO, G::SWZ);
+                        for (int n0 = 0; n0 < len_g[g]; n0 += 256) {   // S[:, range] = K_tile Q_range^T, N <= 256 per MMA
+                            const int nn = len_g[g] - n0 < 256 ? len_g[g] - n0 : 256;
+                            const uint32_t idescS = ptx::instr_desc_bf16(128, nn, 0, 0);
+                            const uint64_t qd = qdesc + (uint64_t)(((c * pl.part_w + n0) * G::RB) >> 4);
+#pragma unroll
+                            for (int k = 0; k < D / 16; ++k)
+                                ptx::mma_ss(buf + c * pl.part_w + n0, kdesc + 2 * k, qd + 2 * k, idescS, k > 0);
+                        }
+                        ptx::mma_commit(bar(S_FULL + g));
+                        if (++s_count[j] == cs) {               // the K tile is free once every range has used it
+                            ptx::mma_commit(bar(K_EMPTY + s));
+                            s_count[j] = 0;
+                        }
+                        ++s_next[g];
+                        v_top[g] = len_g[g];
+                        progressed = true;
+                    } else {                                    // scores issued: feed weights to the value contraction
+                        const int u = v_next[g], len = len_g[g];
+                        const int ho = (len - v_top[g]) / ho_g[g];            // hand-overs go from the top column down
+                        if (!ptx::mbar_test(bar(P_CHUNK + 4 * g + ho), u & 1)) continue;
+                        ptx::tc_fence_after();
+                        const int bottom = v_top[g] - ho_g[g] > 0 ? v_top[g] - ho_g[g] : 0;
+                        const uint32_t dcol = buf + ycol_g[g];
+                        const uint32_t pbase = buf + c * pl.part_w;
+                        const uint64_t zrange = zdesc + (uint64_t)((c * pl.part_w * G::RB) >> 4);
+                        for (int top = v_top[g]; top > bottom;) {           // chunks of 32 score columns (a last one of 16)
+                            const int w = top - bottom >= 32 ? 32 : 16, lo = top - w;
+                            const uint32_t acol = pbase + decode_p_col(len, YC, lo, pl.alias != 0);
+                            for (int sub = 0; sub < w / 16; ++sub) {        // 16 latents: 8 packed columns, 16 rows of Z
+                                const uint64_t bd = zrange + (uint64_t)(((lo + 16 * sub) * G::RB) >> 4);
+                                const uint32_t accum = (top == len && sub == 0) ? 0u : 1u;
+                                ptx::mma_ts(dcol, acol + sub * 8, bd, idescY, accum);
+                                if (!kWide) ptx::mma_ts(dcol, acol + sub * 8, bd + (uint64_t)((M * G::RB) >> 4), idescY, 1u);
+                            }
+                            top = lo;
+                        }
+                        v_top[g] = bottom;
+                        if (bottom == 0) {
+                            ptx::mma_commit(bar(Y_FULL + g));
+                            ++v_next[g];
+                            --remaining;
+                        }
+                        progressed = true;
+                    }
+                }
+                if (progressed) {
+                    spins = 0;
+                } else if ((++spins & 255u) == 0) {             // bounded: give up like every other wait
+                    if (spins == 256u) t0 = ptx::globaltimer_ns();
+                    if (*abort_flag != 0) ok = false;
+                    else if (ptx::globaltimer_ns() - t0 > ptx::kWaitBudgetNs) {
+                        *abort_flag = kErrDecode | 3;
+                        ok = false;
+                    }
                 }
             }
-            if (ok && nbuf == 2 && ntiles > 0) issue_values(ntiles - 1);
         }
-    } else if (warp >= 4) {
-        const int g = (warp - 4) >> 2;                          // softmax group 0 or 1
-        if (g < nbuf) {
-            const int row = ((warp & 3) << 5) + lane;           // TMEM lane = token within the tile
-            const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
-            const uint32_t base = tm + lane_addr + g * cb;
-            for (int i = g; i < ntiles; i += nbuf) {
-                const int u = i / nbuf;
-                if (!warp_wait(bar(S_FULL + g), u & 1, abort_flag, kErrDecode | 6)) break;
-                ptx::tc_fence_after();
-                uint32_t r[32];
-                float mx = -INFINITY;
-                for (int c = 0; c < M / 16; ++c) {              // pass 1: row maximum
-                    ptx::tmem_ld16(base + c * 16, r);
-                    ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) mx = fmaxf(mx, __uint_as_float(r[k]));
-                }
-                const float neg = -mx * a.sl2;
-                float sum = 0.f;
-                for (int c = 0; c < M / 16; ++c) {              // pass 2: exponentials, bf16 pairs over the scores
-                    ptx::tmem_ld16(base + c * 16, r);
-                    ptx::tmem_wait_ld();
-                    uint32_t pk[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const float p0 = ptx::ex2(fmaf(__uint_as_float(r[2 * k]), a.sl2, neg));
-                        const float p1 = ptx::ex2(fmaf(__uint_as_float(r[2 * k + 1]), a.sl2, neg));
-                        sum += p0 + p1;
-                        pk[k] = ptx::pack_bf16(p0, p1);
+    } else if (warp - kFirstSoftmaxWarp < 4 * nbuf * cs) {
+        const int g = (warp - kFirstSoftmaxWarp) >> 2;          // softmax group
+        const int j = g / cs, c = g % cs;                       // its buffer and column range
+        const int row = ((warp & 3) << 5) + lane;               // TMEM lane = token within the tile
+        const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
+        const uint32_t buf = tm + lane_addr + j * cb;
+        const int len = decode_part_len(pl, M, c);
+        const int hcols = decode_handover_cols(len, YC);
+        const bool alias = pl.alias != 0;
+        const uint32_t sbase = buf + c * pl.part_w;             // own scores, and own packed weights over them
+        const float2 sl2p = make_float2(a.sl2, a.sl2);
+        float *my_m = stat_m + g * kTile + row, *my_l = stat_l + g * kTile + row;
+        for (int i = j, u = 0; i < ntiles; i += nbuf, ++u) {
+            if (!warp_wait(bar(S_FULL + g), u & 1, abort_flag, kErrDecode | 6)) break;
+            ptx::tc_fence_after();
+            uint32_t r[32];
+            float mx = -INFINITY;
+            int col = 0;
+            for (; col + 32 <= len; col += 32) {                // pass 1: row maximum over the range
+                ptx::tmem_ld32(sbase + col, r);
+                ptx::tmem_wait_ld();
+                mx = max_of<32>(r, mx);
+            }
+            if (col < len) {
+                ptx::tmem_ld16(sbase + col, r);
+                ptx::tmem_wait_ld();
+                mx = max_of<16>(r, mx);
+            }
+            const float neg = -mx * a.sl2;
+            const float2 negp = make_float2(neg, neg);
+            float2 sum2 = make_float2(0.f, 0.f);
+            uint32_t pk[16];
+            // pass 2, from the top column down: exponentials, bf16 pairs into columns already read (see
+            // decode_p_col); every `hcols` score columns are handed to the value contraction
+            for (int hi = len, ho = 0; hi > 0; ++ho) {
+                const int bottom = hi - hcols > 0 ? hi - hcols : 0;
+                for (int top = hi; top > bottom;) {
+                    if (top - bottom >= 32) {
+                        const int lo = top - 32;
+                        ptx::tmem_ld32(sbase + lo, r);
+                        ptx::tmem_wait_ld();
+                        exp_chunk<32, false>(r, pk, sl2p, negp, sum2);
+                        ptx::tmem_st16(sbase + decode_p_col(len, YC, lo, alias), pk);
+                        top = lo;
+                    } else {
+                        const int lo = top - 16;
+                        ptx::tmem_ld16(sbase + lo, r);
+                        ptx::tmem_wait_ld();
+                        exp_chunk<16, false>(r, pk, sl2p, negp, sum2);
+                        ptx::tmem_st8(sbase + decode_p_col(len, YC, lo, alias), pk);
+                        top = lo;
                     }
-                    ptx::tmem_st8(base + c * 8, pk);
+                }
+                if (bottom == 0 && cs > 1) {                    // statistics travel with the last hand-over
+                    *my_m = mx * a.sl2;
+                    *my_l = sum2.x + sum2.y;
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(bar(P_FULL + g));
-                if (!warp_wait(bar(Y_FULL + g), u & 1, abort_flag, kErrDecode | 7)) break;
-                ptx::tc_fence_after();
-                uint32_t y[D];
+                ptx::mbar_arrive(bar(P_CHUNK + 4 * g + ho));
+                hi = bottom;
+            }
+            const float sum = sum2.x + sum2.y;
+            if (u % cs != c) continue;                          // the ranges take turns writing the tile's rows
+            // every range's statistics are in shared memory once its threads have arrived on its last hand-over,
+            // and its Y accumulator is complete once its Y_FULL has fired
+            bool all = true;
+            for (int cc = 0; cc < cs && all; ++cc) {
+                const int gg = j * cs + cc, lcc = decode_part_len(pl, M, cc);
+                const int last = (lcc + decode_handover_cols(lcc, YC) - 1) / decode_handover_cols(lcc, YC) - 1;
+                all = warp_wait(bar(P_CHUNK + 4 * gg + last), u & 1, abort_flag, kErrDecode | 8) &&
+                      warp_wait(bar(Y_FULL + gg), u & 1, abort_flag, kErrDecode | 7);
+            }
+            if (!all) break;
+            ptx::tc_fence_after();
+            // merge the ranges: weights 2^(m_c - m), total sum l
+            float mtot = mx * a.sl2, ltot = sum, wgt[4] = {1.f, 1.f, 1.f, 1.f};
+            if (cs > 1) {
+                float mc[4], lc[4];
+                mtot = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < D / 16; ++c) ptx::tmem_ld16(base + y_off + c * 16, y + c * 16);
-                ptx::tmem_wait_ld();
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(bar(BUF_EMPTY + g));
-                const int n = (t_begin + i) * kTile + row;
-                if (n < a.N) {
-                    const float inv = 1.f / sum;
-                    uint4 *dst = reinterpret_cast<uint4 *>(a.Y + (((size_t)b * a.N + n) * a.H + h) * D);
+                for (int cc = 0; cc < 4; ++cc) {
+                    mc[cc] = cc < cs ? stat_m[(j * cs + cc) * kTile + row] : -INFINITY;
+                    lc[cc] = cc < cs ? stat_l[(j * cs + cc) * kTile + row] : 0.f;
+                    mtot = fmaxf(mtot, mc[cc]);
+                }
+                ltot = 0.f;
 #pragma unroll
-                    for (int c = 0; c < D / 8; ++c) {
-                        uint4 v;
-                        v.x = ptx::pack_bf16(__uint_as_float(y[c * 8 + 0]) * inv, __uint_as_float(y[c * 8 + 1]) * inv);
-                        v.y = ptx::pack_bf16(__uint_as_float(y[c * 8 + 2]) * inv, __uint_as_float(y[c * 8 + 3]) * inv);
-                        v.z = ptx::pack_bf16(__uint_as_float(y[c * 8 + 4]) * inv, __uint_as_float(y[c * 8 + 5]) * inv);
-                        v.w = ptx::pack_bf16(__uint_as_float(y[c * 8 + 6]) * inv, __uint_as_float(y[c * 8 + 7]) * inv);
-                        dst[c] = v;
-                    }
-                    if (a.lse_dec != nullptr)
-                        a.lse_dec[((size_t)b * a.N + n) * a.H + h] = (mx * a.sl2 + log2f(sum)) * 0.6931471805599453f;
+                for (int cc = 0; cc < 4; ++cc) {
+                    wgt[cc] = ptx::ex2(mc[cc] - mtot);
+                    ltot = fmaf(wgt[cc], lc[cc], ltot);
                 }
             }
+            const float inv = 1.f / ltot;
+            const int n = (t_begin + i) * kTile + row;
+            uint4 *dst = reinterpret_cast<uint4 *>(a.Y + (((size_t)b * a.N + (n < a.N ? n : 0)) * a.H + h) * D);
+#pragma unroll
+            for (int dc = 0; dc < D / 16; ++dc) {
+                float y[16];
+                uint32_t t[16];
+#pragma unroll
+                for (int k = 0; k < 16; ++k) y[k] = 0.f;
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    if (cc < cs) {
+#pragma unroll
+                        for (int half = 0; half < (kWide ? 2 : 1); ++half) {   // wide form: hi and lo products
+                            ptx::tmem_ld16(buf + y_col(cc) + half * D + dc * 16, t);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) y[k] = fmaf(__uint_as_float(t[k]), wgt[cc], y[k]);
+                        }
+                    }
+                }
+                if (n < a.N) {
+                    dst[2 * dc] = make_uint4(ptx::pack_bf16(y[0] * inv, y[1] * inv), ptx::pack_bf16(y[2] * inv, y[3] * inv),
+                                             ptx::pack_bf16(y[4] * inv, y[5] * inv), ptx::pack_bf16(y[6] * inv, y[7] * inv));
+                    dst[2 * dc + 1] =
+                        make_uint4(ptx::pack_bf16(y[8] * inv, y[9] * inv), ptx::pack_bf16(y[10] * inv, y[11] * inv),
+                                   ptx::pack_bf16(y[12] * inv, y[13] * inv), ptx::pack_bf16(y[14] * inv, y[15] * inv));
+                }
+            }
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(bar(BUF_EMPTY + j));
+            if (n < a.N && a.lse_dec != nullptr)
+                a.lse_dec[((size_t)b * a.N + n) * a.H + h] = (mtot + log2f(ltot)) * 0.6931471805599453f;
         }
     }
     // teardown: everyone arrives here (waits are bounded), then the allocating warp frees tensor memory
@@ -274,7 +512,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tm, ncols);
+        ptx::tmem_dealloc(tm, (uint32_t)pl.ncols);
     }
     if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
 }
@@ -290,7 +528,7 @@ struct EncodeTcArgs {
     int tiles;        // ceil(N / 128)
     int splits;       // CTAs along N per (b, h, latent-block pair)
     int pairs;        // ceil(ceil(M/128) / 2)
-    int partials_per_split;  // 2 when M <= 128 (two slots alternate tiles), else 1
+    int partials_per_split;  // 4 when M <= 128 (two slots alternate tiles, two column halves each), else 2
 };
 
 template <int D>
@@ -306,8 +544,10 @@ struct EncodeSmem {
 };
 
 // Encode, split over N.  grid = (splits, H * pairs, B).  A CTA owns up to two blocks of 128 latents of head h
-// ("slots", one softmax group and one TMEM score buffer + accumulator each) and a contiguous range of token
-// tiles.  With M <= 128 the two slots share the one latent block and take alternate tiles.
+// ("slots", one TMEM score buffer each) and a contiguous range of token tiles.  With M <= 128 the two slots
+// share the one latent block and take alternate tiles.  Each slot is served by two softmax groups that split
+// the tile's 128 token columns in halves, each half with its own running maximum, sum and accumulator, i.e.
+// its own partial result for the merge kernel.
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -320,7 +560,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint8_t *sQ = smem + SM::q_off();
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off());
     enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_FULL = S_FULL + 2,
-           ACC_DONE = P_FULL + 2, Q_FULL, NBARS };
+           ACC_DONE = P_FULL + 4, Q_FULL, NBARS };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -337,13 +577,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
     const int rows_here = min(M - lb0 * kTile, 2 * kTile);      // latent rows of Q_h this CTA needs
-    constexpr int SLOT_COLS = 256;                              // per slot: scores/P at [0,128), accumulator at [128,128+D)
+    constexpr int SLOT_COLS = 256;   // per slot: scores / packed weights at [0,128), accumulators at 128 + 64 * half
+    constexpr int HALF = kTile / 2;
     constexpr uint32_t NCOLS = 512;
 
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NBARS; ++i) ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2) ? 128u : 1u);
+        for (int i = 0; i < NBARS; ++i) ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 4) ? 128u : 1u);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
@@ -378,7 +619,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (lane == 0) {
             const uint32_t idescS = ptx::instr_desc_bf16(128, kTile, 0, 0);
             const uint32_t idescV = ptx::instr_desc_bf16(128, D, 0, 1);
-            const uint32_t qaddr = ptx::smem_u32(sQ);
+            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ);
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 2);
             auto tile_of = [&](int q) { return alternate ? q : q / nslots; };
             auto slot_of = [&](int q) { return alternate ? (q & 1) : q % nslots; };
@@ -386,23 +627,31 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int t = tile_of(q), j = slot_of(q), s = t % kEncStages;
                 if (!ptx::mbar_wait(bar(KV_FULL + s), (t / kEncStages) & 1, abort_flag, kErrEncode | 3)) return false;
                 ptx::tc_fence_after();
-                const uint32_t kaddr = ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES);
-                const uint32_t qa = qaddr + (alternate ? 0 : j * kTile * G::RB);
+                const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES), 16, G::SBO, G::SWZ);
+                const uint64_t qa = qdesc + (uint64_t)(alternate ? 0 : j * kTile * G::RB / 16);
+#pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    ptx::mma_ss(tm + j * SLOT_COLS, ptx::smem_desc(qa + k * 32, 16, G::SBO, G::SWZ),
-                                ptx::smem_desc(kaddr + k * 32, 16, G::SBO, G::SWZ), idescS, k > 0);
+                    ptx::mma_ss(tm + j * SLOT_COLS, qa + 2 * k, kdesc + 2 * k, idescS, k > 0);
                 ptx::mma_commit(bar(S_FULL + j));
                 return true;
             };
             auto issue_values = [&](int q) -> bool {
                 const int t = tile_of(q), j = slot_of(q), s = t % kEncStages;
                 const int u = alternate ? (q >> 1) : t;        // how many jobs this slot has done before
-                if (!ptx::mbar_wait(bar(P_FULL + j), u & 1, abort_flag, kErrEncode | 4)) return false;
-                ptx::tc_fence_after();
-                const uint32_t vaddr = ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES);
-                for (int k = 0; k < kTile / 16; ++k)
-                    ptx::mma_ts(tm + j * SLOT_COLS + kTile, tm + j * SLOT_COLS + k * 8,
-                                ptx::smem_desc(vaddr + k * 16 * G::RB, G::SBO, G::SBO, G::SWZ), idescV, (u > 0 || k > 0));
+                // V tile as the MN-major B operand; 16 token rows further on per k-step (descriptor units of 16 bytes)
+                const uint64_t vdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES),
+                                                      G::SBO, G::SBO, G::SWZ);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {                   // the two column halves, each into its own accumulator
+                    if (!ptx::mbar_wait(bar(P_FULL + 2 * j + c), u & 1, abort_flag, kErrEncode | 4)) return false;
+                    ptx::tc_fence_after();
+                    const uint32_t dcol = tm + j * SLOT_COLS + kTile + c * HALF;
+                    const uint32_t acol = tm + j * SLOT_COLS + c * HALF;
+                    const uint64_t bd = vdesc + (uint64_t)(c * HALF * G::RB / 16);
+#pragma unroll
+                    for (int k = 0; k < HALF / 16; ++k)
+                        ptx::mma_ts(dcol, acol + k * 8, bd + (uint64_t)(k * G::RB), idescV, (u > 0 || k > 0));
+                }
                 if (alternate || j == nslots - 1) ptx::mma_commit(bar(KV_EMPTY + s));  // last job of this tile
                 return true;
             };
@@ -414,96 +663,91 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             if (ok) ptx::mma_commit(bar(ACC_DONE));
         }
-    } else if (warp >= 4) {
-        const int g = (warp - 4) >> 2;                          // softmax group = slot
+    } else {
+        const int g = (warp - kFirstSoftmaxWarp) >> 2;          // softmax group
+        const int j = g >> 1, c = g & 1;                        // its slot and column half
         const int row = ((warp & 3) << 5) + lane;               // TMEM lane = latent within the block
         const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
-        const uint32_t sbase = tm + lane_addr + g * SLOT_COLS, abase = sbase + kTile;
-        float m_run = -INFINITY, l_run = 0.f;
+        const uint32_t sbase = tm + lane_addr + j * SLOT_COLS + c * HALF;   // own score columns, own weights over them
+        const uint32_t abase = tm + lane_addr + j * SLOT_COLS + kTile + c * HALF;
+        const float2 sl2p = make_float2(a.sl2, a.sl2);
+        float m_run = -INFINITY;
+        float2 l2 = make_float2(0.f, 0.f);
         int done = 0;
         bool ok = true;
-        if (g < nslots) {
-            for (int q = g; q < nq; q += nslots, ++done) {
+        if (j < nslots) {
+            for (int q = j; q < nq; q += nslots, ++done) {
                 const int t = t_begin + (alternate ? q : q / nslots);
-                // validity bits of the tile's 128 tokens (tail beyond N, padding mask), one word per 32 tokens
-                uint32_t wv[4];
+                // validity bits of this half's 64 tokens (tail beyond N, padding mask), one word per 32 tokens
+                uint32_t wv[2];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int n = t * kTile + c * 32 + lane;
+                for (int w = 0; w < 2; ++w) {
+                    const int n = t * kTile + c * HALF + w * 32 + lane;
                     const bool valid = n < a.N && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0);
-                    wv[c] = __ballot_sync(0xffffffffu, valid);
+                    wv[w] = __ballot_sync(0xffffffffu, valid);
                 }
-                const uint32_t w0 = wv[0], w1 = wv[1], w2 = wv[2], w3 = wv[3];
-                const bool all_valid = (w0 & w1 & w2 & w3) == 0xffffffffu;
-                if (!warp_wait(bar(S_FULL + g), done & 1, abort_flag, kErrEncode | 5)) { ok = false; break; }
+                const uint32_t w0 = wv[0], w1 = wv[1];
+                const bool all_valid = (w0 & w1) == 0xffffffffu;
+                if (!warp_wait(bar(S_FULL + j), done & 1, abort_flag, kErrEncode | 5)) { ok = false; break; }
                 ptx::tc_fence_after();
                 uint32_t r[32];
                 float tmax = -INFINITY;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {                   // pass 1: tile maximum over valid tokens
-                    ptx::tmem_ld32(sbase + c * 32, r);
+                for (int w = 0; w < 2; ++w) {                   // pass 1: maximum over this half's valid tokens
+                    ptx::tmem_ld32(sbase + w * 32, r);
                     ptx::tmem_wait_ld();
-                    const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
                     if (all_valid) {
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) tmax = fmaxf(tmax, __uint_as_float(r[k]));
+                        tmax = max_of<32>(r, tmax);
                     } else {
+                        const uint32_t wm = w == 0 ? w0 : w1;
 #pragma unroll
                         for (int k = 0; k < 32; ++k)
-                            if ((w >> k) & 1) tmax = fmaxf(tmax, __uint_as_float(r[k]));
+                            if ((wm >> k) & 1) tmax = fmaxf(tmax, __uint_as_float(r[k]));
                     }
                 }
                 const float m_new = fmaxf(m_run, tmax);
                 const bool grow = done > 0 && m_new > m_run;
                 if (__any_sync(0xffffffffu, grow)) {            // rescale the accumulator row (warp-uniform branch)
                     const float f = grow ? ptx::ex2((m_run - m_new) * a.sl2) : 1.f;
-                    l_run *= f;
+                    l2.x *= f;
+                    l2.y *= f;
 #pragma unroll
-                    for (int c = 0; c < D / 16; ++c) {
-                        ptx::tmem_ld16(abase + c * 16, r);
+                    for (int dc = 0; dc < D / 16; ++dc) {
+                        ptx::tmem_ld16(abase + dc * 16, r);
                         ptx::tmem_wait_ld();
 #pragma unroll
                         for (int k = 0; k < 16; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) * f);
-                        ptx::tmem_st16(abase + c * 16, r);
+                        ptx::tmem_st16(abase + dc * 16, r);
                     }
                 }
                 m_run = m_new;
                 const bool dead = (m_run == -INFINITY);         // no valid token yet: all weights are zero
                 const float neg = dead ? 0.f : -m_run * a.sl2;
+                const float2 negp = make_float2(neg, neg);
+                uint32_t pk[16];
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {                   // pass 2: weights, bf16 pairs over the scores
-                    ptx::tmem_ld32(sbase + c * 32, r);
+                for (int w = 0; w < 2; ++w) {                   // pass 2: weights, bf16 pairs over the scores
+                    ptx::tmem_ld32(sbase + w * 32, r);
                     ptx::tmem_wait_ld();
-                    const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        float p0 = ptx::ex2(fmaf(__uint_as_float(r[2 * k]), a.sl2, neg));
-                        float p1 = ptx::ex2(fmaf(__uint_as_float(r[2 * k + 1]), a.sl2, neg));
-                        if (!all_valid) {
-                            if (dead || !((w >> (2 * k)) & 1)) p0 = 0.f;
-                            if (dead || !((w >> (2 * k + 1)) & 1)) p1 = 0.f;
-                        }
-                        l_run += p0 + p1;
-                        pk[k] = ptx::pack_bf16(p0, p1);
-                    }
-                    ptx::tmem_st16(sbase + c * 16, pk);
+                    if (all_valid) exp_chunk<32, false>(r, pk, sl2p, negp, l2);
+                    else exp_chunk<32, true>(r, pk, sl2p, negp, l2, w == 0 ? w0 : w1, dead);
+                    ptx::tmem_st16(sbase + w * 16, pk);
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(bar(P_FULL + g));
+                ptx::mbar_arrive(bar(P_FULL + 2 * j + c));
             }
         }
-        // write this slot's partial (running max in natural-log units, sum, un-normalised rows)
+        // write this group's partial (running max in natural-log units, sum, un-normalised rows)
         if (ok) ok = warp_wait(bar(ACC_DONE), 0, abort_flag, kErrEncode | 6);
         ptx::tc_fence_after();
-        const int lb = alternate ? 0 : lb0 + g;
+        const int lb = alternate ? 0 : lb0 + j;
         const int m = lb * kTile + row;
-        const bool writes = ok && (alternate || g < nslots);
+        const bool writes = ok && j < nslots;
         uint32_t acc[D];
         if (done > 0) {
 #pragma unroll
-            for (int c = 0; c < D / 16; ++c) ptx::tmem_ld16(abase + c * 16, acc + c * 16);
+            for (int dc = 0; dc < D / 16; ++dc) ptx::tmem_ld16(abase + dc * 16, acc + dc * 16);
             ptx::tmem_wait_ld();
         } else {
 #pragma unroll
@@ -511,14 +755,15 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         if (writes && m < M) {
             const long rows = (long)a.B * a.H * M;
-            const size_t prow = (size_t)(alternate ? split * 2 + g : split) * rows + ((size_t)b * a.H + h) * M + m;
+            const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);
+            const size_t prow = (size_t)part * rows + ((size_t)b * a.H + h) * M + m;
             a.part_m[prow] = (m_run == -INFINITY) ? -INFINITY : m_run * a.scale;
-            a.part_l[prow] = l_run;
+            a.part_l[prow] = l2.x + l2.y;
             float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * D);
 #pragma unroll
-            for (int c = 0; c < D / 4; ++c)
-                dst[c] = make_float4(__uint_as_float(acc[4 * c]), __uint_as_float(acc[4 * c + 1]),
-                                     __uint_as_float(acc[4 * c + 2]), __uint_as_float(acc[4 * c + 3]));
+            for (int dc = 0; dc < D / 4; ++dc)
+                dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
+                                      __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
         }
     }
     ptx::tc_fence_before();
