@@ -11,11 +11,14 @@
 // (latent, token) pair needs one exponential on the special-function unit (16 per clock per SM), and every
 // tcgen05.mma of this shape (M = 128, K = 16) holds the tensor pipe for about 107 cycles whatever its N
 // (measured), so the value contraction costs one such slot per 16 latents (decode) or tokens (encode): about
-// as long as the exponentials of the same block.  The CTA is built to keep both busy at once: warp 0 issues
-// TMA loads, warp 1 issues the MMAs and owns the TMEM allocation, and sixteen softmax warps (four per
-// scheduler) form four groups of four warps.  A group owns one TMEM score buffer, or a range of columns of a
-// shared one, with its own running maximum, sum and accumulator columns; while one group waits for its MMAs
-// the other three keep the schedulers fed.
+// as long as the exponentials of the same block.  That cost is a latency of the issuing thread, not an occupancy
+// of the pipe: four threads issuing side by side get about three times the instructions through (measured).
+// The CTA is therefore four pipelines side by side: warp 0 issues TMA loads; sixteen softmax warps (four per
+// scheduler) form four groups of four warps, and each group has an issuing warp of its own (warps 1-4; warp 1
+// also owns the TMEM allocation).  A group owns one TMEM score buffer, or a range of columns of a shared one,
+// with its own score MMA, running maximum, sum and accumulator columns; its weights go to its value
+// contraction a few columns at a time as they are written.  While one group waits for its MMAs the other
+// three keep the schedulers and the special-function unit fed.
 #pragma once
 
 #include "flare_common.cuh"
@@ -24,8 +27,9 @@
 namespace flare {
 
 constexpr int kSoftmaxGroups = 4;                            // groups of 4 warps (128 threads = 128 TMEM lanes)
-constexpr int kFirstSoftmaxWarp = 2;
-constexpr int kTcThreads = (kFirstSoftmaxWarp + 4 * kSoftmaxGroups) * 32;  // 576
+constexpr int kFirstIssuerWarp = 1;                          // warps 1..4: one MMA-issuing warp per group
+constexpr int kFirstSoftmaxWarp = kFirstIssuerWarp + kSoftmaxGroups;
+constexpr int kTcThreads = (kFirstSoftmaxWarp + 4 * kSoftmaxGroups) * 32;  // 672
 constexpr int kTile = 128;       // tokens per tile (decode: TMEM lanes; encode: score columns)
 constexpr int kDecStages = 4;    // K tiles in flight (decode)
 constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode)
@@ -228,14 +232,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBARS; ++i) {
             const bool counted = (i >= P_CHUNK && i < P_CHUNK + 4 * NG) || (i >= BUF_EMPTY && i < BUF_EMPTY + NG);
-            ptx::mbar_init(bar(i), counted ? 128u : 1u);
+            const bool per_range = i >= K_EMPTY && i < K_EMPTY + kDecStages;   // every range's issuer releases the K tile
+            ptx::mbar_init(bar(i), counted ? 128u : per_range ? (uint32_t)cs : 1u);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
         ptx::prefetch_tensormap(&tmQ);
     }
-    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), (uint32_t)pl.ncols);
+    if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), (uint32_t)pl.ncols);
     // Z_bh -> two bf16 halves (hi = round(z), lo = round(z - hi)); rows of RB bytes in the swizzled layout the
     // MMA's B operand expects (latent-major rows), the lo half M rows after the hi half.
     {
@@ -278,105 +283,54 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                  (t_begin + i) * kTile, b);
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            // The MMA thread is a scheduler over the groups' pipelines: for each group it issues, whichever is
-            // ready, the scores of the group's next tile (K tile landed, buffer drained) or the value contraction of
-            // the next columns of weights the group has handed over.
+    } else if (warp < kFirstSoftmaxWarp) {
+        const int g = warp - kFirstIssuerWarp;                  // the group this warp issues MMAs for
+        if (lane == 0 && g < nbuf * cs) {
+            // One issuing thread per group: the scores of the group's next tile as soon as its K tile has landed and
+            // its buffer is drained, then the value contraction of each hand-over of weights as it arrives.
+            const int j = g / cs, c = g % cs;
+            const int len = decode_part_len(pl, M, c), hcols = decode_handover_cols(len, YC);
             const uint32_t idescY = ptx::instr_desc_bf16(128, YC, 0, 1);
-            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ);
-            // Z as the MN-major B operand: 8-row groups SBO apart; in the wide form the lo half is the second block
-            // along N, M rows further on.  Descriptor address fields are in 16-byte units.
+            // Q rows of this range (K-major B operand of the score MMA); descriptor address fields are in 16-byte units
+            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ) + (uint64_t)((c * pl.part_w * G::RB) >> 4);
+            // Z rows of this range as the MN-major B operand: 8-row groups SBO apart; in the wide form the lo half is
+            // the second block along N, M rows further on
             const uint64_t zdesc = ptx::smem_desc(ptx::smem_u32(sZ), kWide ? (uint32_t)(M * G::RB) : (uint32_t)G::SBO,
-                                                  G::SBO, G::SWZ);
-            const int ng = nbuf * cs;
-            int len_g[NG], ycol_g[NG], ho_g[NG];                // per group: range length, Y column, columns per hand-over
-            int s_next[NG], v_next[NG], v_top[NG];              // per group: tiles whose scores / values are issued; columns left
-            int s_count[NG];                                    // per buffer: ranges of the current tile whose scores are issued
-#pragma unroll
-            for (int g = 0; g < NG; ++g) {
-                const int c = g % cs;
-                len_g[g] = g < ng ? decode_part_len(pl, M, c) : 0;
-                ycol_g[g] = g < ng ? y_col(c) : 0;
-                ho_g[g] = decode_handover_cols(len_g[g], YC);
-                s_next[g] = v_next[g] = v_top[g] = s_count[g] = 0;
-            }
+                                                  G::SBO, G::SWZ) + (uint64_t)((c * pl.part_w * G::RB) >> 4);
+            const uint32_t sbuf = tm + j * cb + c * pl.part_w;  // the range's scores / packed weights
+            const uint32_t dcol = tm + j * cb + y_col(c);
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrDecode | 2);
-            int remaining = 0;                                  // (group, tile) pairs still to finish
-            for (int g = 0; g < ng; ++g) remaining += (ntiles - g / cs + nbuf - 1) / nbuf;
-            uint64_t t0 = 0;                                    // start of the current stretch without progress
-            uint32_t spins = 0;
-            while (ok && remaining > 0) {
-                bool progressed = false;
+            for (int i = j, u = 0; ok && i < ntiles; i += nbuf, ++u) {
+                const int s = i % nstages;
+                if (!ptx::mbar_wait(bar(K_FULL + s), (i / nstages) & 1, abort_flag, kErrDecode | 3)) break;
+                if (!ptx::mbar_wait(bar(BUF_EMPTY + j), (u & 1) ^ 1, abort_flag, kErrDecode | 4)) break;
+                ptx::tc_fence_after();
+                const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), 16, G::SBO, G::SWZ);
+                for (int n0 = 0; n0 < len; n0 += 256) {         // S[:, range] = K_tile Q_range^T, N <= 256 per MMA
+                    const int nn = len - n0 < 256 ? len - n0 : 256;
+                    const uint32_t idescS = ptx::instr_desc_bf16(128, nn, 0, 0);
+                    const uint64_t qd = qdesc + (uint64_t)((n0 * G::RB) >> 4);
 #pragma unroll
-                for (int g = 0; g < NG; ++g) {
-                    if (g >= ng) break;
-                    const int j = g / cs, c = g % cs;
-                    const uint32_t buf = tm + j * cb;
-                    if (s_next[g] == v_next[g]) {               // idle: try to issue the scores of the group's next tile
-                        const int u = s_next[g], i = j + u * nbuf;
-                        if (i >= ntiles) continue;
-                        const int s = i % nstages;
-                        if (!ptx::mbar_test(bar(K_FULL + s), (i / nstages) & 1) ||
-                            !ptx::mbar_test(bar(BUF_EMPTY + j), (u & 1) ^ 1))
-                            continue;
-                        ptx::tc_fence_after();
-                        const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), 16, G::SBO, G::SWZ);
-                        for (int n0 = 0; n0 < len_g[g]; n0 += 256) {   // S[:, range] = K_tile Q_range^T, N <= 256 per MMA
-                            const int nn = len_g[g] - n0 < 256 ? len_g[g] - n0 : 256;
-                            const uint32_t idescS = ptx::instr_desc_bf16(128, nn, 0, 0);
-                            const uint64_t qd = qdesc + (uint64_t)(((c * pl.part_w + n0) * G::RB) >> 4);
-#pragma unroll
-                            for (int k = 0; k < D / 16; ++k)
-                                ptx::mma_ss(buf + c * pl.part_w + n0, kdesc + 2 * k, qd + 2 * k, idescS, k > 0);
+                    for (int k = 0; k < D / 16; ++k) ptx::mma_ss(sbuf + n0, kdesc + 2 * k, qd + 2 * k, idescS, k > 0);
+                }
+                ptx::mma_commit(bar(S_FULL + g));
+                ptx::mma_commit(bar(K_EMPTY + s));              // one arrival per range: the K tile is free after the last
+                for (int top = len, ho = 0; ok && top > 0; ++ho) {   // hand-overs go from the top column down
+                    if (!ptx::mbar_wait(bar(P_CHUNK + 4 * g + ho), u & 1, abort_flag, kErrDecode | 5)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const int bottom = top - hcols > 0 ? top - hcols : 0;
+                    while (top > bottom) {                      // chunks of 32 score columns (a last one of 16)
+                        const int w = top - bottom >= 32 ? 32 : 16, lo = top - w;
+                        const uint32_t acol = sbuf + decode_p_col(len, YC, lo, pl.alias != 0);
+                        for (int sub = 0; sub < w / 16; ++sub) {    // 16 latents: 8 packed columns, 16 rows of Z
+                            const uint64_t bd = zdesc + (uint64_t)(((lo + 16 * sub) * G::RB) >> 4);
+                            ptx::mma_ts(dcol, acol + sub * 8, bd, idescY, (top == len && sub == 0) ? 0u : 1u);
+                            if (!kWide) ptx::mma_ts(dcol, acol + sub * 8, bd + (uint64_t)((M * G::RB) >> 4), idescY, 1u);
                         }
-                        ptx::mma_commit(bar(S_FULL + g));
-                        if (++s_count[j] == cs) {               // the K tile is free once every range has used it
-                            ptx::mma_commit(bar(K_EMPTY + s));
-                            s_count[j] = 0;
-                        }
-                        ++s_next[g];
-                        v_top[g] = len_g[g];
-                        progressed = true;
-                    } else {                                    // scores issued: feed weights to the value contraction
-                        const int u = v_next[g], len = len_g[g];
-                        const int ho = (len - v_top[g]) / ho_g[g];            // hand-overs go from the top column down
-                        if (!ptx::mbar_test(bar(P_CHUNK + 4 * g + ho), u & 1)) continue;
-                        ptx::tc_fence_after();
-                        const int bottom = v_top[g] - ho_g[g] > 0 ? v_top[g] - ho_g[g] : 0;
-                        const uint32_t dcol = buf + ycol_g[g];
-                        const uint32_t pbase = buf + c * pl.part_w;
-                        const uint64_t zrange = zdesc + (uint64_t)((c * pl.part_w * G::RB) >> 4);
-                        for (int top = v_top[g]; top > bottom;) {           // chunks of 32 score columns (a last one of 16)
-                            const int w = top - bottom >= 32 ? 32 : 16, lo = top - w;
-                            const uint32_t acol = pbase + decode_p_col(len, YC, lo, pl.alias != 0);
-                            for (int sub = 0; sub < w / 16; ++sub) {        // 16 latents: 8 packed columns, 16 rows of Z
-                                const uint64_t bd = zrange + (uint64_t)(((lo + 16 * sub) * G::RB) >> 4);
-                                const uint32_t accum = (top == len && sub == 0) ? 0u : 1u;
-                                ptx::mma_ts(dcol, acol + sub * 8, bd, idescY, accum);
-                                if (!kWide) ptx::mma_ts(dcol, acol + sub * 8, bd + (uint64_t)((M * G::RB) >> 4), idescY, 1u);
-                            }
-                            top = lo;
-                        }
-                        v_top[g] = bottom;
-                        if (bottom == 0) {
-                            ptx::mma_commit(bar(Y_FULL + g));
-                            ++v_next[g];
-                            --remaining;
-                        }
-                        progressed = true;
+                        top = lo;
                     }
                 }
-                if (progressed) {
-                    spins = 0;
-                } else if ((++spins & 255u) == 0) {             // bounded: give up like every other wait
-                    if (spins == 256u) t0 = ptx::globaltimer_ns();
-                    if (*abort_flag != 0) ok = false;
-                    else if (ptx::globaltimer_ns() - t0 > ptx::kWaitBudgetNs) {
-                        *abort_flag = kErrDecode | 3;
-                        ok = false;
-                    }
-                }
+                if (ok) ptx::mma_commit(bar(Y_FULL + g));
             }
         }
     } else if (warp - kFirstSoftmaxWarp < 4 * nbuf * cs) {
@@ -510,7 +464,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // teardown: everyone arrives here (waits are bounded), then the allocating warp frees tensor memory
     ptx::tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kFirstIssuerWarp) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tm, (uint32_t)pl.ncols);
     }
@@ -546,8 +500,8 @@ struct EncodeSmem {
 // Encode, split over N.  grid = (splits, H * pairs, B).  A CTA owns up to two blocks of 128 latents of head h
 // ("slots", one TMEM score buffer each) and a contiguous range of token tiles.  With M <= 128 the two slots
 // share the one latent block and take alternate tiles.  Each slot is served by two softmax groups that split
-// the tile's 128 token columns in halves, each half with its own running maximum, sum and accumulator, i.e.
-// its own partial result for the merge kernel.
+// the tile's 128 token columns in halves; a half is a pipeline of its own, with its own issuing warp, score
+// MMA (N = 64), running maximum, sum and accumulator, i.e. its own partial result for the merge kernel.
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -559,8 +513,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint8_t *sKV = smem + SM::kv_off;
     uint8_t *sQ = smem + SM::q_off();
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off());
-    enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_FULL = S_FULL + 2,
-           ACC_DONE = P_FULL + 4, Q_FULL, NBARS };
+    constexpr int NG = kSoftmaxGroups;
+    // S_FULL, ACC_DONE: one per group; P_CHUNK: two hand-overs (32 token columns each) per group
+    enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_CHUNK = S_FULL + NG,
+           ACC_DONE = P_CHUNK + 2 * NG, Q_FULL = ACC_DONE + NG, NBARS };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -584,14 +540,18 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NBARS; ++i) ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 4) ? 128u : 1u);
+        // a K/V tile is released by the issuers of all the groups that use it
+        const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
+        for (int i = 0; i < NBARS; ++i)
+            ptx::mbar_init(bar(i), (i >= P_CHUNK && i < P_CHUNK + 2 * NG) ? 128u
+                                   : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users : 1u);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
         ptx::prefetch_tensormap(&tmV);
         ptx::prefetch_tensormap(&tmQ);
     }
-    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), NCOLS);
+    if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), NCOLS);
     // latent rows beyond M are zero so their (discarded) lanes stay finite
     for (int i = threadIdx.x; i < (2 * kTile - rows_here) * (G::RB / 16); i += kTcThreads)
         reinterpret_cast<uint4 *>(sQ + (size_t)rows_here * G::RB)[i] = make_uint4(0, 0, 0, 0);
@@ -615,53 +575,43 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * D, (t_begin + i) * kTile, b);
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idescS = ptx::instr_desc_bf16(128, kTile, 0, 0);
+    } else if (warp < kFirstSoftmaxWarp) {
+        const int g = warp - kFirstIssuerWarp;                  // the group this warp issues MMAs for
+        const int j = g >> 1, c = g & 1;                        // its slot and column half
+        if (lane == 0 && j < nslots) {
+            const uint32_t idescS = ptx::instr_desc_bf16(128, HALF, 0, 0);
             const uint32_t idescV = ptx::instr_desc_bf16(128, D, 0, 1);
-            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ);
+            // Q rows of the slot's latent block (K-major A operand); descriptor address fields are in 16-byte units
+            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ) +
+                                   (uint64_t)(alternate ? 0 : j * kTile * G::RB / 16);
+            const uint32_t scol = tm + j * SLOT_COLS + c * HALF;            // the half's scores / packed weights
+            const uint32_t dcol = tm + j * SLOT_COLS + kTile + c * HALF;    // its accumulator
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 2);
-            auto tile_of = [&](int q) { return alternate ? q : q / nslots; };
-            auto slot_of = [&](int q) { return alternate ? (q & 1) : q % nslots; };
-            auto issue_scores = [&](int q) -> bool {
-                const int t = tile_of(q), j = slot_of(q), s = t % kEncStages;
-                if (!ptx::mbar_wait(bar(KV_FULL + s), (t / kEncStages) & 1, abort_flag, kErrEncode | 3)) return false;
+            int done = 0;
+            for (int q = j; ok && q < nq; q += nslots, ++done) {
+                const int t = alternate ? q : q / nslots, s = t % kEncStages;
+                if (!ptx::mbar_wait(bar(KV_FULL + s), (t / kEncStages) & 1, abort_flag, kErrEncode | 3)) break;
                 ptx::tc_fence_after();
-                const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES), 16, G::SBO, G::SWZ);
-                const uint64_t qa = qdesc + (uint64_t)(alternate ? 0 : j * kTile * G::RB / 16);
+                const uint32_t kv = ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES);
+                // S[:, half] = Q_block K_half^T: the half's 64 token rows of the K tile are the B operand
+                const uint64_t kdesc = ptx::smem_desc(kv, 16, G::SBO, G::SWZ) + (uint64_t)(c * HALF * G::RB / 16);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k)
-                    ptx::mma_ss(tm + j * SLOT_COLS, qa + 2 * k, kdesc + 2 * k, idescS, k > 0);
-                ptx::mma_commit(bar(S_FULL + j));
-                return true;
-            };
-            auto issue_values = [&](int q) -> bool {
-                const int t = tile_of(q), j = slot_of(q), s = t % kEncStages;
-                const int u = alternate ? (q >> 1) : t;        // how many jobs this slot has done before
-                // V tile as the MN-major B operand; 16 token rows further on per k-step (descriptor units of 16 bytes)
-                const uint64_t vdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES),
-                                                      G::SBO, G::SBO, G::SWZ);
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(scol, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                ptx::mma_commit(bar(S_FULL + g));
+                // acc += P_half V_half: V tile as the MN-major B operand, 16 token rows further on per k-step
+                const uint64_t vdesc = ptx::smem_desc(kv + G::TILE_BYTES, G::SBO, G::SBO, G::SWZ) + (uint64_t)(c * HALF * G::RB / 16);
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {                   // the two column halves, each into its own accumulator
-                    if (!ptx::mbar_wait(bar(P_FULL + 2 * j + c), u & 1, abort_flag, kErrEncode | 4)) return false;
+                for (int w = 0; w < 2; ++w) {                   // hand-overs of 32 token columns
+                    if (!ptx::mbar_wait(bar(P_CHUNK + 2 * g + w), done & 1, abort_flag, kErrEncode | 4)) { ok = false; break; }
                     ptx::tc_fence_after();
-                    const uint32_t dcol = tm + j * SLOT_COLS + kTile + c * HALF;
-                    const uint32_t acol = tm + j * SLOT_COLS + c * HALF;
-                    const uint64_t bd = vdesc + (uint64_t)(c * HALF * G::RB / 16);
 #pragma unroll
-                    for (int k = 0; k < HALF / 16; ++k)
-                        ptx::mma_ts(dcol, acol + k * 8, bd + (uint64_t)(k * G::RB), idescV, (u > 0 || k > 0));
+                    for (int k = 0; k < 2; ++k)
+                        ptx::mma_ts(dcol, scol + w * 16 + k * 8, vdesc + (uint64_t)((2 * w + k) * G::RB), idescV,
+                                    (done > 0 || w > 0 || k > 0) ? 1u : 0u);
                 }
-                if (alternate || j == nslots - 1) ptx::mma_commit(bar(KV_EMPTY + s));  // last job of this tile
-                return true;
-            };
-            const int stride = nslots;
-            for (int q = 0; ok && q < stride && q < nq; ++q) ok = issue_scores(q);
-            for (int q = 0; ok && q < nq; ++q) {
-                ok = issue_values(q);
-                if (ok && q + stride < nq) ok = issue_scores(q + stride);
+                if (ok) ptx::mma_commit(bar(KV_EMPTY + s));     // one arrival per group that used the tile
             }
-            if (ok) ptx::mma_commit(bar(ACC_DONE));
+            if (ok) ptx::mma_commit(bar(ACC_DONE + g));
         }
     } else {
         const int g = (warp - kFirstSoftmaxWarp) >> 2;          // softmax group
@@ -688,7 +638,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 const uint32_t w0 = wv[0], w1 = wv[1];
                 const bool all_valid = (w0 & w1) == 0xffffffffu;
-                if (!warp_wait(bar(S_FULL + j), done & 1, abort_flag, kErrEncode | 5)) { ok = false; break; }
+                if (!warp_wait(bar(S_FULL + g), done & 1, abort_flag, kErrEncode | 5)) { ok = false; break; }
                 ptx::tc_fence_after();
                 uint32_t r[32];
                 float tmax = -INFINITY;
@@ -732,14 +682,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (all_valid) exp_chunk<32, false>(r, pk, sl2p, negp, l2);
                     else exp_chunk<32, true>(r, pk, sl2p, negp, l2, w == 0 ? w0 : w1, dead);
                     ptx::tmem_st16(sbase + w * 16, pk);
+                    ptx::tmem_wait_st();                        // hand these 32 columns to the value contraction
+                    ptx::tc_fence_before();
+                    ptx::mbar_arrive(bar(P_CHUNK + 2 * g + w));
                 }
-                ptx::tmem_wait_st();
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(bar(P_FULL + 2 * j + c));
             }
         }
         // write this group's partial (running max in natural-log units, sum, un-normalised rows)
-        if (ok) ok = warp_wait(bar(ACC_DONE), 0, abort_flag, kErrEncode | 6);
+        if (ok && j < nslots) ok = warp_wait(bar(ACC_DONE + g), 0, abort_flag, kErrEncode | 6);
         ptx::tc_fence_after();
         const int lb = alternate ? 0 : lb0 + j;
         const int m = lb * kTile + row;
@@ -768,7 +718,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     ptx::tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kFirstIssuerWarp) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tm, NCOLS);
     }
