@@ -21,6 +21,8 @@
 // three keep the schedulers and the special-function unit fed.
 #pragma once
 
+#include <type_traits>
+
 #include "flare_common.cuh"
 #include "flare_ptx.cuh"
 
@@ -500,8 +502,11 @@ struct EncodeSmem {
 // Encode, split over N.  grid = (splits, H * pairs, B).  A CTA owns up to two blocks of 128 latents of head h
 // ("slots", one TMEM score buffer each) and a contiguous range of token tiles.  With M <= 128 the two slots
 // share the one latent block and take alternate tiles.  Each slot is served by two softmax groups that split
-// the tile's 128 token columns in halves; a half is a pipeline of its own, with its own issuing warp, score
-// MMA (N = 64), running maximum, sum and accumulator, i.e. its own partial result for the merge kernel.
+// the tile's 128 token columns in halves; a half is a pipeline of its own, with its own issuing warp, running
+// maximum, sum and accumulator, i.e. its own partial result for the merge kernel.  A half is worked off in
+// units of 32 tokens on two alternating score buffers: while the group evaluates the exponentials of one
+// unit, the score MMA of the next and the value MMAs of the previous one run, so that the group never waits
+// for the tensor pipe in steady state.
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -514,9 +519,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint8_t *sQ = smem + SM::q_off();
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off());
     constexpr int NG = kSoftmaxGroups;
-    // S_FULL, ACC_DONE: one per group; P_CHUNK: two hand-overs (32 token columns each) per group
-    enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_CHUNK = S_FULL + NG,
-           ACC_DONE = P_CHUNK + 2 * NG, Q_FULL = ACC_DONE + NG, NBARS };
+    // per group: S_FULL and P_FULL for each of its two score buffers, PV_DONE (one phase per unit), ACC_DONE
+    enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_FULL = S_FULL + 2 * NG,
+           PV_DONE = P_FULL + 2 * NG, ACC_DONE = PV_DONE + NG, Q_FULL = ACC_DONE + NG, NBARS };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -533,8 +538,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
     const int rows_here = min(M - lb0 * kTile, 2 * kTile);      // latent rows of Q_h this CTA needs
-    constexpr int SLOT_COLS = 256;   // per slot: scores / packed weights at [0,128), accumulators at 128 + 64 * half
+    constexpr int SLOT_COLS = 256;   // per slot and half (128 columns): two score buffers of UNIT columns, accumulator at 64
     constexpr int HALF = kTile / 2;
+    constexpr int UNIT = 32;         // tokens per unit of work of a group
     constexpr uint32_t NCOLS = 512;
 
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
@@ -543,7 +549,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // a K/V tile is released by the issuers of all the groups that use it
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
-            ptx::mbar_init(bar(i), (i >= P_CHUNK && i < P_CHUNK + 2 * NG) ? 128u
+            ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? 128u
                                    : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users : 1u);
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -579,37 +585,51 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int g = warp - kFirstIssuerWarp;                  // the group this warp issues MMAs for
         const int j = g >> 1, c = g & 1;                        // its slot and column half
         if (lane == 0 && j < nslots) {
-            const uint32_t idescS = ptx::instr_desc_bf16(128, HALF, 0, 0);
+            const uint32_t idescS = ptx::instr_desc_bf16(128, UNIT, 0, 0);
             const uint32_t idescV = ptx::instr_desc_bf16(128, D, 0, 1);
             // Q rows of the slot's latent block (K-major A operand); descriptor address fields are in 16-byte units
             const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ) +
                                    (uint64_t)(alternate ? 0 : j * kTile * G::RB / 16);
-            const uint32_t scol = tm + j * SLOT_COLS + c * HALF;            // the half's scores / packed weights
-            const uint32_t dcol = tm + j * SLOT_COLS + kTile + c * HALF;    // its accumulator
+            const uint32_t gcol = tm + j * SLOT_COLS + c * 2 * HALF;        // the group's 128 columns
+            const uint32_t dcol = gcol + 2 * UNIT;                          // its accumulator
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 2);
-            int done = 0;
-            for (int q = j; ok && q < nq; q += nslots, ++done) {
-                const int t = alternate ? q : q / nslots, s = t % kEncStages;
-                if (!ptx::mbar_wait(bar(KV_FULL + s), (t / kEncStages) & 1, abort_flag, kErrEncode | 3)) break;
+            const int jobs = (nq - j + nslots - 1) / nslots;                // tiles this group works on
+            const int units = 2 * jobs;
+            // Order of issue: S(0), S(1), then for every unit n: its value MMAs as soon as its weights are handed
+            // over, then the scores of unit n+2 into the buffer those weights have just left.  Every wait blocks
+            // in hardware, so the issuing warp takes no issue slots from the softmax warps while it waits.
+            int t_s = alternate ? j : 0, t_v = t_s;                         // tiles (relative to t_begin) of the next S / PV unit
+            const int t_step = alternate ? 2 : 1;
+            auto issue_scores = [&](int n) -> bool {
+                const int s = t_s % kEncStages, w = n & 1;                  // w: which 32 tokens of the half; also the buffer
+                if (!ptx::mbar_wait(bar(KV_FULL + s), (t_s / kEncStages) & 1, abort_flag, kErrEncode | 3)) return false;
                 ptx::tc_fence_after();
-                const uint32_t kv = ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES);
-                // S[:, half] = Q_block K_half^T: the half's 64 token rows of the K tile are the B operand
-                const uint64_t kdesc = ptx::smem_desc(kv, 16, G::SBO, G::SWZ) + (uint64_t)(c * HALF * G::RB / 16);
+                // S_unit = Q_block K_unit^T: the unit's 32 token rows of the K tile are the B operand
+                const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES), 16, G::SBO, G::SWZ) +
+                                       (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(scol, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
-                ptx::mma_commit(bar(S_FULL + g));
-                // acc += P_half V_half: V tile as the MN-major B operand, 16 token rows further on per k-step
-                const uint64_t vdesc = ptx::smem_desc(kv + G::TILE_BYTES, G::SBO, G::SBO, G::SWZ) + (uint64_t)(c * HALF * G::RB / 16);
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                ptx::mma_commit(bar(S_FULL + 2 * g + w));
+                if (w == 1) t_s += t_step;
+                return true;
+            };
+            for (int n = 0; ok && n < 2 && n < units; ++n) ok = issue_scores(n);
+            for (int n = 0; ok && n < units; ++n) {
+                const int w = n & 1, s = t_v % kEncStages;
+                if (!ptx::mbar_wait(bar(P_FULL + 2 * g + w), (n >> 1) & 1, abort_flag, kErrEncode | 4)) break;
+                ptx::tc_fence_after();
+                // acc += P_unit V_unit: V tile as the MN-major B operand, 16 token rows further on per k-step
+                const uint64_t vdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES),
+                                                      G::SBO, G::SBO, G::SWZ) + (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
 #pragma unroll
-                for (int w = 0; w < 2; ++w) {                   // hand-overs of 32 token columns
-                    if (!ptx::mbar_wait(bar(P_CHUNK + 2 * g + w), done & 1, abort_flag, kErrEncode | 4)) { ok = false; break; }
-                    ptx::tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < 2; ++k)
-                        ptx::mma_ts(dcol, scol + w * 16 + k * 8, vdesc + (uint64_t)((2 * w + k) * G::RB), idescV,
-                                    (done > 0 || w > 0 || k > 0) ? 1u : 0u);
+                for (int k = 0; k < UNIT / 16; ++k)
+                    ptx::mma_ts(dcol, gcol + w * UNIT + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, (n > 0 || k > 0) ? 1u : 0u);
+                ptx::mma_commit(bar(PV_DONE + g));
+                if (w == 1) {                                               // the tile's last unit: one arrival per group
+                    ptx::mma_commit(bar(KV_EMPTY + s));
+                    t_v += t_step;
                 }
-                if (ok) ptx::mma_commit(bar(KV_EMPTY + s));     // one arrival per group that used the tile
+                if (n + 2 < units) ok = issue_scores(n + 2);
             }
             if (ok) ptx::mma_commit(bar(ACC_DONE + g));
         }
@@ -618,74 +638,75 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int j = g >> 1, c = g & 1;                        // its slot and column half
         const int row = ((warp & 3) << 5) + lane;               // TMEM lane = latent within the block
         const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
-        const uint32_t sbase = tm + lane_addr + j * SLOT_COLS + c * HALF;   // own score columns, own weights over them
-        const uint32_t abase = tm + lane_addr + j * SLOT_COLS + kTile + c * HALF;
+        const uint32_t gcol = tm + lane_addr + j * SLOT_COLS + c * 2 * HALF;   // the group's 128 columns
+        const uint32_t abase = gcol + 2 * UNIT;                               // its accumulator
         const float2 sl2p = make_float2(a.sl2, a.sl2);
         float m_run = -INFINITY;
         float2 l2 = make_float2(0.f, 0.f);
-        int done = 0;
+        int done = 0;                                           // units finished
         bool ok = true;
-        if (j < nslots) {
-            for (int q = j; q < nq; q += nslots, ++done) {
-                const int t = t_begin + (alternate ? q : q / nslots);
-                // validity bits of this half's 64 tokens (tail beyond N, padding mask), one word per 32 tokens
-                uint32_t wv[2];
+        // One unit of work: 32 token columns of this group's half, on score buffer w.  kMasked: some of the tile's
+        // tokens may be padding or lie beyond N (their weights are exactly 0); the plain form has no such tests.
+        auto unit = [&](auto masked, int t, int w) -> bool {
+            constexpr bool kMasked = decltype(masked)::value;
+            uint32_t wv = 0xffffffffu;
+            if (kMasked) {
+                const int n = t * kTile + c * HALF + w * UNIT + lane;
+                wv = __ballot_sync(0xffffffffu, n < a.N && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0));
+            }
+            const uint32_t sbase = gcol + w * UNIT;             // the unit's scores, and its packed weights over them
+            if (!warp_wait(bar(S_FULL + 2 * g + w), (done >> 1) & 1, abort_flag, kErrEncode | 5)) return false;
+            ptx::tc_fence_after();
+            uint32_t r[32];
+            ptx::tmem_ld32(sbase, r);                           // the scores stay in registers for both passes
+            ptx::tmem_wait_ld();
+            float tmax = -INFINITY;
+            if (!kMasked) {
+                tmax = max_of<32>(r, tmax);
+            } else {
 #pragma unroll
-                for (int w = 0; w < 2; ++w) {
-                    const int n = t * kTile + c * HALF + w * 32 + lane;
-                    const bool valid = n < a.N && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0);
-                    wv[w] = __ballot_sync(0xffffffffu, valid);
-                }
-                const uint32_t w0 = wv[0], w1 = wv[1];
-                const bool all_valid = (w0 & w1) == 0xffffffffu;
-                if (!warp_wait(bar(S_FULL + g), done & 1, abort_flag, kErrEncode | 5)) { ok = false; break; }
+                for (int k = 0; k < 32; ++k)
+                    if ((wv >> k) & 1) tmax = fmaxf(tmax, __uint_as_float(r[k]));
+            }
+            const float m_new = fmaxf(m_run, tmax);
+            const bool grow = done > 0 && m_new > m_run;
+            if (__any_sync(0xffffffffu, grow)) {                // rescale the accumulator row (warp-uniform branch)
+                // the value MMAs of every earlier unit must have landed in the accumulator first
+                if (!warp_wait(bar(PV_DONE + g), (done - 1) & 1, abort_flag, kErrEncode | 7)) return false;
                 ptx::tc_fence_after();
-                uint32_t r[32];
-                float tmax = -INFINITY;
-#pragma unroll 1
-                for (int w = 0; w < 2; ++w) {                   // pass 1: maximum over this half's valid tokens
-                    ptx::tmem_ld32(sbase + w * 32, r);
+                const float f = grow ? ptx::ex2((m_run - m_new) * a.sl2) : 1.f;
+                l2.x *= f;
+                l2.y *= f;
+                uint32_t ar[16];
+#pragma unroll
+                for (int dc = 0; dc < D / 16; ++dc) {
+                    ptx::tmem_ld16(abase + dc * 16, ar);
                     ptx::tmem_wait_ld();
-                    if (all_valid) {
-                        tmax = max_of<32>(r, tmax);
-                    } else {
-                        const uint32_t wm = w == 0 ? w0 : w1;
 #pragma unroll
-                        for (int k = 0; k < 32; ++k)
-                            if ((wm >> k) & 1) tmax = fmaxf(tmax, __uint_as_float(r[k]));
-                    }
+                    for (int k = 0; k < 16; ++k) ar[k] = __float_as_uint(__uint_as_float(ar[k]) * f);
+                    ptx::tmem_st16(abase + dc * 16, ar);
                 }
-                const float m_new = fmaxf(m_run, tmax);
-                const bool grow = done > 0 && m_new > m_run;
-                if (__any_sync(0xffffffffu, grow)) {            // rescale the accumulator row (warp-uniform branch)
-                    const float f = grow ? ptx::ex2((m_run - m_new) * a.sl2) : 1.f;
-                    l2.x *= f;
-                    l2.y *= f;
-#pragma unroll
-                    for (int dc = 0; dc < D / 16; ++dc) {
-                        ptx::tmem_ld16(abase + dc * 16, r);
-                        ptx::tmem_wait_ld();
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) r[k] = __float_as_uint(__uint_as_float(r[k]) * f);
-                        ptx::tmem_st16(abase + dc * 16, r);
-                    }
-                }
-                m_run = m_new;
-                const bool dead = (m_run == -INFINITY);         // no valid token yet: all weights are zero
-                const float neg = dead ? 0.f : -m_run * a.sl2;
-                const float2 negp = make_float2(neg, neg);
-                uint32_t pk[16];
+            }
+            m_run = m_new;
+            const bool dead = (m_run == -INFINITY);             // no valid token yet: all weights are zero
+            const float neg = dead ? 0.f : -m_run * a.sl2;
+            const float2 negp = make_float2(neg, neg);
+            uint32_t pk[16];
+            exp_chunk<32, kMasked>(r, pk, sl2p, negp, l2, wv, dead);
+            ptx::tmem_st16(sbase, pk);
+            ptx::tmem_wait_st();                                // weights (and a rescaled accumulator) are in place
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(bar(P_FULL + 2 * g + w));
+            ++done;
+            return true;
+        };
+        if (j < nslots) {
+            for (int q = j; ok && q < nq; q += nslots) {
+                const int t = t_begin + (alternate ? q : q / nslots);
+                const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;   // warp-uniform
 #pragma unroll 1
-                for (int w = 0; w < 2; ++w) {                   // pass 2: weights, bf16 pairs over the scores
-                    ptx::tmem_ld32(sbase + w * 32, r);
-                    ptx::tmem_wait_ld();
-                    if (all_valid) exp_chunk<32, false>(r, pk, sl2p, negp, l2);
-                    else exp_chunk<32, true>(r, pk, sl2p, negp, l2, w == 0 ? w0 : w1, dead);
-                    ptx::tmem_st16(sbase + w * 16, pk);
-                    ptx::tmem_wait_st();                        // hand these 32 columns to the value contraction
-                    ptx::tc_fence_before();
-                    ptx::mbar_arrive(bar(P_CHUNK + 2 * g + w));
-                }
+                for (int w = 0; ok && w < 2; ++w)               // the half's two units, on alternating buffers
+                    ok = plain ? unit(std::false_type{}, t, w) : unit(std::true_type{}, t, w);
             }
         }
         // write this group's partial (running max in natural-log units, sum, un-normalised rows)
