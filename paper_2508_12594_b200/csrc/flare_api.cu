@@ -110,12 +110,15 @@ struct TcEncodePlan {
     int tiles, pairs, splits, per_split, P;
 };
 
+// With at most 64 latents a CTA encodes two adjacent heads at once (see encode_tc_kernel).
+bool encode_head_pairs(const flare_desc_t *d) { return d->M <= 64 && d->H % 2 == 0 && d->D <= 32; }
+
 TcEncodePlan tc_encode_plan(const flare_desc_t *d, int sms) {
     TcEncodePlan p;
     p.tiles = (d->N + kTile - 1) / kTile;
     const int mb = (d->M + kTile - 1) / kTile;
     p.pairs = (mb + 1) / 2;
-    long groups = (long)d->B * d->H * p.pairs;
+    long groups = (long)d->B * (encode_head_pairs(d) ? d->H / 2 : d->H) * p.pairs;
     long s = sms / groups;
     if (s < 1) s = 1;
     if (s > p.tiles) s = p.tiles;
@@ -148,8 +151,10 @@ CUtensorMapSwizzle swizzle_for(int D) {
     return D == 16 ? CU_TENSOR_MAP_SWIZZLE_32B : D == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
 }
 
-// [B, N, H*D] bf16 viewed as a 3-D tensor (innermost H*D); box = one head's D columns x `rows` tokens.
-int make_token_map(CUtensorMap *m, const void *base, const flare_desc_t *d, int rows) {
+// [B, N, H*D] bf16 viewed as a 3-D tensor (innermost H*D); box = `cols` columns (one head's D, or two adjacent
+// heads' 2D) x `rows` tokens.
+int make_token_map(CUtensorMap *m, const void *base, const flare_desc_t *d, int rows, int cols = 0) {
+    if (cols == 0) cols = d->D;
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) {
         snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled not available");
@@ -158,10 +163,10 @@ int make_token_map(CUtensorMap *m, const void *base, const flare_desc_t *d, int 
     const cuuint64_t C = (cuuint64_t)d->H * d->D;
     cuuint64_t dims[3] = {C, (cuuint64_t)d->N, (cuuint64_t)d->B};
     cuuint64_t strides[2] = {C * 2, C * 2 * (cuuint64_t)d->N};
-    cuuint32_t box[3] = {(cuuint32_t)d->D, (cuuint32_t)rows, 1};
+    cuuint32_t box[3] = {(cuuint32_t)cols, (cuuint32_t)rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(d->D), CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(cols), CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled(tokens) failed: %d", (int)r);
@@ -193,27 +198,29 @@ int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int D>
+template <int D, bool kPair>
 int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
                      const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st) {
+    constexpr int DG = kPair ? 2 * D : D;
     CUtensorMap tmK, tmV, tmQ;
     int rc;
-    if ((rc = make_token_map(&tmK, K, d, kTile)) != FLARE_OK) return rc;
-    if ((rc = make_token_map(&tmV, V, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmK, K, d, kTile, DG)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmV, V, d, kTile, DG)) != FLARE_OK) return rc;
     if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
-    const size_t smem = EncodeSmem<D>::total();
+    const size_t smem = EncodeSmem<DG>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     EncodeTcArgs a;
+    a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.key_mask = mask; a.part_m = pm; a.part_l = pl; a.part_acc = pacc; a.status = status;
     a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
-    dim3 grid(p.splits, d->H * p.pairs, d->B);
-    encode_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
+    encode_tc_kernel<D, kPair><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -390,9 +397,13 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
     if (use_tc(d)) {
         TcEncodePlan p = tc_encode_plan(d, di.sms);
         uint32_t *status = reinterpret_cast<uint32_t *>(base);
-        rc = d->D == 16   ? launch_encode_tc<16>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-             : d->D == 32 ? launch_encode_tc<32>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-                          : launch_encode_tc<64>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
+        if (encode_head_pairs(d))
+            rc = d->D == 16 ? launch_encode_tc<16, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+                            : launch_encode_tc<32, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
+        else
+            rc = d->D == 16   ? launch_encode_tc<16, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+                 : d->D == 32 ? launch_encode_tc<32, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+                              : launch_encode_tc<64, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
     } else {
         SimtPlan p = simt_plan(d, di.sms);
         rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)

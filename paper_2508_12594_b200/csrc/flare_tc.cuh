@@ -476,6 +476,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 // ------------------------------------------------------------------------------------------------ encode
 
 struct EncodeTcArgs {
+    const __nv_bfloat16 *Q;   // [H,M,D] (read directly in the head-pair form)
     const uint8_t *key_mask;  // [B,N] or null
     float *part_m, *part_l, *part_acc;
     uint32_t *status;
@@ -487,9 +488,10 @@ struct EncodeTcArgs {
     int partials_per_split;  // 4 when M <= 128 (two slots alternate tiles, two column halves each), else 2
 };
 
-template <int D>
+// DG: columns of a K/V tile row as the kernel sees it (D, or 2D in the head-pair form).
+template <int DG>
 struct EncodeSmem {
-    using G = TileGeom<D>;
+    using G = TileGeom<DG>;
     static constexpr size_t kv_off = 0;                         // [stage][K tile | V tile]
     __host__ __device__ static size_t q_off() { return (size_t)kEncStages * 2 * G::TILE_BYTES; }
     __host__ __device__ static size_t bar_off() { return q_off() + (size_t)2 * kTile * G::RB; }
@@ -507,12 +509,19 @@ struct EncodeSmem {
 // units of 32 tokens on two alternating score buffers: while the group evaluates the exponentials of one
 // unit, the score MMA of the next and the value MMAs of the previous one run, so that the group never waits
 // for the tensor pipe in steady state.
-template <int D>
+//
+// Head-pair form (kPair; M <= 64, H even, D <= 32): with at most 64 latents half of the 128 lanes would idle, so
+// a CTA takes two adjacent heads at once.  Lanes 0-63 hold the latents of head 2p, lanes 64-127 those of head
+// 2p+1; the A operand is the block-diagonal [Q_2p 0; 0 Q_2p+1] over the 2D feature columns the two heads occupy
+// side by side in a token row, so one MMA with K = 2D gives every lane its own head's scores, and the value MMA
+// with N = 2D gives lanes 0-63 their rows in accumulator columns [0, D) and lanes 64-127 theirs in [D, 2D).
+template <int D, bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
-    using G = TileGeom<D>;
-    using SM = EncodeSmem<D>;
+    constexpr int DG = kPair ? 2 * D : D;
+    using G = TileGeom<DG>;
+    using SM = EncodeSmem<DG>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sKV = smem + SM::kv_off;
@@ -527,7 +536,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int M = a.M;
-    const int split = blockIdx.x, h = blockIdx.y / a.pairs, pair = blockIdx.y % a.pairs, b = blockIdx.z;
+    // h: the head, or in the head-pair form the first head of the pair
+    const int split = blockIdx.x, h = (kPair ? 2 : 1) * (blockIdx.y / a.pairs), pair = blockIdx.y % a.pairs, b = blockIdx.z;
     const int t_begin = (int)((long)a.tiles * split / a.splits);
     const int t_end = (int)((long)a.tiles * (split + 1) / a.splits);
     const int nt = t_end - t_begin;
@@ -537,7 +547,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int lb0 = pair * 2;                                   // latent block of slot 0
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
-    const int rows_here = min(M - lb0 * kTile, 2 * kTile);      // latent rows of Q_h this CTA needs
+    const int rows_here = kPair ? 0 : min(M - lb0 * kTile, 2 * kTile);   // latent rows of Q_h fetched by TMA
     constexpr int SLOT_COLS = 256;   // per slot and half (128 columns): two score buffers of UNIT columns, accumulator at 64
     constexpr int HALF = kTile / 2;
     constexpr int UNIT = 32;         // tokens per unit of work of a group
@@ -561,6 +571,16 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // latent rows beyond M are zero so their (discarded) lanes stay finite
     for (int i = threadIdx.x; i < (2 * kTile - rows_here) * (G::RB / 16); i += kTcThreads)
         reinterpret_cast<uint4 *>(sQ + (size_t)rows_here * G::RB)[i] = make_uint4(0, 0, 0, 0);
+    if (kPair) {
+        // block-diagonal A operand: row r < 64 = [Q[h][r] | 0], row 64 + r = [0 | Q[h+1][r]], 16-byte chunks swizzled
+        __syncthreads();
+        for (int i = threadIdx.x; i < 2 * M * (D / 8); i += kTcThreads) {
+            const int which = i / (M * (D / 8)), rem = i % (M * (D / 8)), m = rem / (D / 8), ch = rem % (D / 8);
+            const uint4 v = *reinterpret_cast<const uint4 *>(a.Q + ((size_t)(h + which) * M + m) * D + ch * 8);
+            const int r = which * 64 + m, chunk = which * (D / 8) + ch;
+            *reinterpret_cast<uint4 *>(sQ + (size_t)r * G::RB + ((chunk ^ G::swz(r)) << 4)) = v;
+        }
+    }
     ptx::fence_proxy_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
@@ -569,9 +589,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(rows_here * G::RB));
-            for (int r = 0; r < rows_here; r += 16)
-                ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
+            if (kPair) {
+                ptx::mbar_arrive(bar(Q_FULL));                  // Q was written by the threads before the block barrier
+            } else {
+                ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(rows_here * G::RB));
+                for (int r = 0; r < rows_here; r += 16)
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
+            }
             for (int i = 0; i < nt; ++i) {
                 const int s = i % kEncStages;
                 if (!ptx::mbar_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
@@ -586,7 +610,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int j = g >> 1, c = g & 1;                        // its slot and column half
         if (lane == 0 && j < nslots) {
             const uint32_t idescS = ptx::instr_desc_bf16(128, UNIT, 0, 0);
-            const uint32_t idescV = ptx::instr_desc_bf16(128, D, 0, 1);
+            const uint32_t idescV = ptx::instr_desc_bf16(128, DG, 0, 1);
             // Q rows of the slot's latent block (K-major A operand); descriptor address fields are in 16-byte units
             const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ) +
                                    (uint64_t)(alternate ? 0 : j * kTile * G::RB / 16);
@@ -608,7 +632,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES), 16, G::SBO, G::SWZ) +
                                        (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                for (int k = 0; k < DG / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
                 ptx::mma_commit(bar(S_FULL + 2 * g + w));
                 if (w == 1) t_s += t_step;
                 return true;
@@ -679,7 +703,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 l2.y *= f;
                 uint32_t ar[16];
 #pragma unroll
-                for (int dc = 0; dc < D / 16; ++dc) {
+                for (int dc = 0; dc < DG / 16; ++dc) {
                     ptx::tmem_ld16(abase + dc * 16, ar);
                     ptx::tmem_wait_ld();
 #pragma unroll
@@ -713,12 +737,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (ok && j < nslots) ok = warp_wait(bar(ACC_DONE + g), 0, abort_flag, kErrEncode | 6);
         ptx::tc_fence_after();
         const int lb = alternate ? 0 : lb0 + j;
-        const int m = lb * kTile + row;
+        // head-pair form: lanes 64-127 belong to the second head, whose rows are accumulator columns [D, 2D)
+        const int second = kPair ? (row >> 6) : 0;
+        const int m = kPair ? (row & 63) : lb * kTile + row;
         const bool writes = ok && j < nslots;
         uint32_t acc[D];
         if (done > 0) {
 #pragma unroll
-            for (int dc = 0; dc < D / 16; ++dc) ptx::tmem_ld16(abase + dc * 16, acc + dc * 16);
+            for (int dc = 0; dc < D / 16; ++dc) ptx::tmem_ld16(abase + second * D + dc * 16, acc + dc * 16);
             ptx::tmem_wait_ld();
         } else {
 #pragma unroll
@@ -727,7 +753,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (writes && m < M) {
             const long rows = (long)a.B * a.H * M;
             const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);
-            const size_t prow = (size_t)part * rows + ((size_t)b * a.H + h) * M + m;
+            const size_t prow = (size_t)part * rows + ((size_t)b * a.H + h + second) * M + m;
             a.part_m[prow] = (m_run == -INFINITY) ? -INFINITY : m_run * a.scale;
             a.part_l[prow] = l2.x + l2.y;
             float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * D);
