@@ -45,7 +45,7 @@ EDGE = [
     (2, 1, 300, 256, 64, "bf16", 0.0),
     (1, 1, 515, 512, 16, "bf16", 0.5),
     (1, 2, 1000, 80, 32, "bf16", 0.0),
-    (2, 3, 700, 32, 16, "bf16", 0.2),      # odd head count: one head per CTA although M <= 64
+    (2, 3, 1100, 32, 16, "bf16", 0.2),     # odd head count: one head per CTA although M <= 64
     (1, 4, 900, 16, 16, "bf16", 0.0),      # two heads per CTA, most latent lanes empty
     (1, 6, 450, 64, 32, "bf16", 0.3),      # two heads per CTA, all lanes in use, padding
     (3, 2, 333, 5, 32, "f32", 0.4),
