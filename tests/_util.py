@@ -17,6 +17,32 @@ def rel_err(got, ref):
     return float(np.abs(got - ref).max()) / max(rms, 1e-300)
 
 
+def bf16_round(x):
+    """The float64 array rounded to bfloat16 (round to nearest even) and widened again."""
+    return torch.from_numpy(np.asarray(x, dtype=np.float64)).float().bfloat16().double().numpy()
+
+
+def assert_stored_close(got, ref, dtype, what):
+    """The bound on a tensor that is stored in the call dtype.
+
+    The stated bound is max|err| <= tol * RMS(ref).  For a bfloat16 tensor it cannot hold for entries larger than
+    about 5 RMS whatever the kernel does: rounding the exact value to bfloat16 is an error of up to 2^-8 |ref|,
+    which passes 2e-2 RMS at |ref| = 5.12 RMS (the mesh workloads have entries of 8 RMS and more; the oracle's own
+    Y rounded to bfloat16 breaks the stated bound there, see test_oracle_pins.py).  So the stated bound is tried
+    first, and where it fails the bound is the stated one plus exactly one rounding of the stored value:
+    |err| <= tol * RMS(ref) + 2^-8 |ref|, element by element."""
+    tol = TOL[dtype]
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = max(float(np.sqrt(np.mean(ref ** 2))), 1e-300)
+    err = np.abs(got - ref)
+    if err.max() <= tol * rms:
+        return
+    assert dtype == "bf16", f"{what}: max|err|/RMS = {err.max() / rms:.3e} > {tol}"
+    excess = (err - 2.0 ** -8 * np.abs(ref)).max() / rms
+    assert excess <= tol, f"{what}: (max|err| - one bf16 rounding)/RMS = {excess:.3e} > {tol}"
+
+
 def to_np64(t):
     return None if t is None else t.double().cpu().numpy()
 
@@ -61,9 +87,9 @@ def oracle_forward(oracle, inp, scale=1.0):
 
 def assert_forward_close(got, ref, dtype, what=""):
     tol = TOL[dtype]
-    for name in ("Z", "Y"):
-        e = rel_err(got[name], ref[name])
-        assert e <= tol, f"{what} {name}: max|err|/RMS = {e:.3e} > {tol}"
+    e = rel_err(got["Z"], ref["Z"])                      # Z is float32 in memory: the stated bound as it stands
+    assert e <= tol, f"{what} Z: max|err|/RMS = {e:.3e} > {tol}"
+    assert_stored_close(got["Y"], ref["Y"], dtype, f"{what} Y")
     for name in ("lse_enc", "lse_dec"):
         fin = np.isfinite(ref[name])
         assert np.array_equal(np.isneginf(got[name]), np.isneginf(ref[name])), f"{what} {name}: -inf pattern"

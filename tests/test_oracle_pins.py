@@ -248,6 +248,20 @@ def test_backward_value_gradient_sums(oracle):
     assert (g["dV"][mask == 0] == 0).all()
 
 
+def test_bf16_storage_alone_can_break_the_stated_bound(oracle):
+    """On the mesh workload the exact Y has entries of many RMS; rounding the oracle's own Y to bfloat16 is then by
+    itself an error above 2e-2 RMS(Y) at full size.  This is why the GPU tests allow one rounding of the stored
+    value on top of the stated bound where the stated bound fails."""
+    w = workloads.CONFIGS["mesh2d"].with_(B=1, N=16384)
+    Q, K, V, _, _ = _np(workloads.make_inputs(w))
+    Y = oracle.forward(Q, K, V)["Y"]
+    Yb = torch.from_numpy(Y).float().bfloat16().double().numpy()
+    rms = np.sqrt(np.mean(Y ** 2))
+    assert np.abs(Y).max() > 5.12 * rms
+    assert np.abs(Yb - Y).max() > 1.5e-2 * rms           # storage rounding alone takes most or all of the stated 2e-2
+    assert (np.abs(Yb - Y) <= 2.0 ** -8 * np.abs(Y)).all()
+
+
 def test_workload_recipes_are_seeded():
     w = workloads.CONFIGS["tiny"]
     a, b = workloads.make_inputs(w), workloads.make_inputs(w)
