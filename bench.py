@@ -29,6 +29,11 @@ from paper_2508_12594_b200 import workloads  # noqa: E402
 
 METRIC = "FLARE fwd tokens/sec at N=1M on 1 B200"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (read + write) of one launch of each main kernel on the full mesh3d_1m workload, from the ncu captures
+# summarised under profiles/ (taken on a 262,144-token slice and scaled by 4: traffic is proportional to N).
+# Valid for the kernels as profiled; set to None when a kernel changes until the capture is redone.
+NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.322432e6 + 4.238592e6),
+               ("mesh3d_1m", "decode"): 4 * (68.100864e6 + 31.640320e6)}
 
 
 def get_workload(name: str) -> workloads.Workload:
@@ -137,13 +142,13 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="mesh3d_1m")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-tokens", type=int, default=32768, help="tokens per batch item in the oracle sample")
-    ap.add_argument("--ref-tokens", type=int, default=16384)
+    ap.add_argument("--cpu-tokens", type=int, default=524288, help="tokens per batch item in the oracle sample")
+    ap.add_argument("--ref-tokens", type=int, default=65536)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override N (a smaller case of the same workload)")
@@ -288,8 +293,14 @@ def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_by
     else:
         roof = {"bound": "hbm", "achieved": bytes_stage / t_dom / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update({"traffic": None, "kernel": dom, "kernel_ms": stage_ms[dom], "peak_kind": peak_kind,
-                 "stage_ms": stage_ms, "exp_per_s": w.B * w.H * w.N * w.M / t_dom})
+    base_name = w.name.split("@")[0]
+    traffic = NCU_TRAFFIC.get((base_name, dom))
+    if traffic is not None:
+        traffic *= w.N / workloads.CONFIGS[base_name].N       # a --tokens slice of the profiled workload
+    sm_clock = (clocks or {}).get("sm_mhz") or 1965.0
+    roof.update({"traffic": traffic, "kernel": dom, "kernel_ms": stage_ms[dom], "peak_kind": peak_kind,
+                 "stage_ms": stage_ms, "exp_per_s": w.B * w.H * w.N * w.M / t_dom,
+                 "exp_per_clk_per_sm": w.B * w.H * w.N * w.M / t_dom / 148 / (sm_clock * 1e6)})
     # whole forward against the stated roofline: slower of 8*B*H*N*M*D FLOP at tensor peak and K, V, Q_lat, Y once
     fwd_t = max(2 * flops_stage / (tensor_peak * 1e12), (3 * tensor_bytes + w.H * w.M * w.D * e) / (peaks["hbm_gbs"] * 1e9))
     roof["forward_frac_of_stated_roofline"] = fwd_t / (ms_step / 1e3)
