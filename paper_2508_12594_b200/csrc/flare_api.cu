@@ -198,9 +198,11 @@ int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int D, bool kPair>
+// kDz: the backward's dZ form of the kernel (V is then dY, lse_dec the decode log-sum-exp rows, pm and pl unused).
+template <int D, bool kPair, bool kDz = false>
 int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
-                     const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st) {
+                     const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
+                     const float *lse_dec = nullptr) {
     constexpr int DG = kPair ? 2 * D : D;
     CUtensorMap tmK, tmV, tmQ;
     int rc;
@@ -210,17 +212,18 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     const size_t smem = EncodeSmem<DG>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     EncodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
+    a.lse_dec = lse_dec;
     a.key_mask = mask; a.part_m = pm; a.part_l = pl; a.part_acc = pacc; a.status = status;
     a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -292,6 +295,9 @@ int launch_decode_simt(const flare_desc_t *d, const void *Q, const void *K, cons
 
 // Launch plans of the CUDA-core backward: pass A (dZ) reuses the encode plan; the dQ pass keeps three latent
 // rows per thread in shared memory and therefore caps its latent block at 64.
+// Pass A (dZ) runs as the dZ form of the tensor-core encode kernel wherever that kernel runs.
+bool bwd_dz_on_tensor_cores(const flare_desc_t *d) { return use_tc(d); }
+
 SimtPlan bwd_dq_plan(const flare_desc_t *d, int sms) {
     SimtPlan p = simt_plan(d, sms);
     if (p.LM > 64) p.LM = 64;
@@ -310,6 +316,7 @@ BwdLayout bwd_layout(const flare_desc_t *d, int sms) {
     const long rows = (long)d->B * d->H * d->M;
     const int pa = simt_plan(d, sms).P, pb = bwd_dq_plan(d, sms).P;
     w.P = pa > pb ? pa : pb;
+    if (bwd_dz_on_tensor_cores(d) && tc_encode_plan(d, sms).P > w.P) w.P = tc_encode_plan(d, sms).P;
     size_t off = kHeaderBytes;
     w.part = off; off += align_up(sizeof(float) * (size_t)w.P * rows * d->D);
     w.dz = off;   off += align_up(sizeof(float) * (size_t)rows * d->D);
@@ -332,10 +339,33 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     const long rows = (long)d->B * d->H * d->M;
     const SimtPlan pa = simt_plan(d, sms), pb = bwd_dq_plan(d, sms);
     FLARE_CUDA(cudaMemsetAsync(ws, 0, kHeaderBytes, st));
-    bwd_dz_simt_kernel<T, D><<<dim3(pa.splits, d->H, d->B), kBwdThreads, 0, st>>>(
-        (const T *)Q, (const T *)K, (const T *)dY, lse_dec, part, d->B, d->H, d->N, d->M, pa.LM, pa.chunk, d->scale);
+    int dz_parts = pa.P;
+    bool dz_on_tc = false;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && (D == 16 || D == 32 || D == 64)) {
+        if (bwd_dz_on_tensor_cores(d)) {
+            const TcEncodePlan tp = tc_encode_plan(d, sms);
+            uint32_t *status = reinterpret_cast<uint32_t *>(ws);
+            int rc;
+            if constexpr (D <= 32) {
+                rc = encode_head_pairs(d)
+                         ? launch_encode_tc<D, true, true>(d, tp, Q, K, dY, nullptr, nullptr, nullptr, part, status, st, lse_dec)
+                         : launch_encode_tc<D, false, true>(d, tp, Q, K, dY, nullptr, nullptr, nullptr, part, status, st, lse_dec);
+            } else {
+                rc = launch_encode_tc<D, false, true>(d, tp, Q, K, dY, nullptr, nullptr, nullptr, part, status, st, lse_dec);
+            }
+            if (rc != FLARE_OK) return rc;
+            dz_parts = tp.P;
+            dz_on_tc = true;
+        }
+    }
+    if (!dz_on_tc) {
+        bwd_dz_simt_kernel<T, D><<<dim3(pa.splits, d->H, d->B), kBwdThreads, 0, st>>>(
+            (const T *)Q, (const T *)K, (const T *)dY, lse_dec, part, d->B, d->H, d->N, d->M, pa.LM, pa.chunk, d->scale);
+        FLARE_CUDA(cudaGetLastError());
+    }
+    bwd_dz_reduce_kernel<<<(unsigned)((rows * d->D + 255) / 256), 256, 0, st>>>(part, dZ, dz_parts, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
-    bwd_dz_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(part, Z, dZ, de, pa.P, rows, d->D);
+    bwd_de_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(dZ, Z, de, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
     bwd_token_simt_kernel<T, D><<<dim3((d->N + 127) / 128, d->H, d->B), 128, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, lse_enc, lse_dec, (T *)dK, (T *)dV, dd,

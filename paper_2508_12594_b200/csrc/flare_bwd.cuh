@@ -75,19 +75,23 @@ bwd_dz_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
     }
 }
 
-// dZ[row][d] = sum_p part[p][row][d];  de[row] = dZ_row . Z_row.  One thread per row.
+// dZ[row][d] = sum_p part[p][row][d], partials added in index order.  One thread per (row, d).
 __global__ void __launch_bounds__(256)
-bwd_dz_reduce_kernel(const float *__restrict__ part, const float *__restrict__ Z, float *__restrict__ dZ,
-                     float *__restrict__ de, int P, long rows, int D) {
+bwd_dz_reduce_kernel(const float *__restrict__ part, float *__restrict__ dZ, int P, long rows, int D) {
+    const long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * D) return;
+    float s = 0.f;
+    for (int p = 0; p < P; ++p) s += part[(size_t)p * rows * D + idx];
+    dZ[idx] = s;
+}
+
+// de[row] = dZ_row . Z_row.  One thread per row.
+__global__ void __launch_bounds__(256)
+bwd_de_kernel(const float *__restrict__ dZ, const float *__restrict__ Z, float *__restrict__ de, long rows, int D) {
     const long row = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= rows) return;
     float dot = 0.f;
-    for (int d = 0; d < D; ++d) {
-        float s = 0.f;
-        for (int p = 0; p < P; ++p) s += part[((size_t)p * rows + row) * D + d];
-        dZ[row * D + d] = s;
-        dot = fmaf(s, Z[row * D + d], dot);
-    }
+    for (int d = 0; d < D; ++d) dot = fmaf(dZ[row * D + d], Z[row * D + d], dot);
     de[row] = dot;
 }
 

@@ -58,6 +58,28 @@ struct TileGeom {
 };
 
 // ------------------------------------------------------------------------------------- softmax arithmetic
+// p = 2^(s * sl2 + neg[k]) with one addend per column (read from shared memory, four at a time): the form the
+// backward needs, where every column (token) carries its own log-sum-exp.  The weights leave as two bf16 halves,
+// hi = round(p) and lo = round(p - hi): dZ feeds differences (dZ.V - dZ.Z) downstream, and with one half its
+// rounding alone moved dK, dV and dQ by 2e-2 to 4e-2 of their RMS (measured).
+template <int NV>
+__device__ __forceinline__ void exp_chunk_cols(const uint32_t *r, uint32_t *hi, uint32_t *lo, float2 sl2p, const float *neg) {
+#pragma unroll
+    for (int k = 0; k < NV / 4; ++k) {
+        const float4 ng = *reinterpret_cast<const float4 *>(neg + 4 * k);
+        const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(r[4 * k]), __uint_as_float(r[4 * k + 1])), sl2p,
+                                     make_float2(ng.x, ng.y));
+        const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(r[4 * k + 2]), __uint_as_float(r[4 * k + 3])), sl2p,
+                                     make_float2(ng.z, ng.w));
+        const float p0 = ptx::ex2(x0.x), p1 = ptx::ex2(x0.y), p2 = ptx::ex2(x1.x), p3 = ptx::ex2(x1.y);
+        const uint32_t h0 = ptx::pack_bf16(p0, p1), h1 = ptx::pack_bf16(p2, p3);
+        hi[2 * k] = h0;
+        hi[2 * k + 1] = h1;
+        lo[2 * k] = ptx::pack_bf16(p0 - __uint_as_float(h0 << 16), p1 - __uint_as_float(h0 & 0xffff0000u));
+        lo[2 * k + 1] = ptx::pack_bf16(p2 - __uint_as_float(h1 << 16), p3 - __uint_as_float(h1 & 0xffff0000u));
+    }
+}
+
 // Row maximum over NV (16 or 32) float32 scores held as raw bits.
 template <int NV>
 __device__ __forceinline__ float max_of(const uint32_t *r, float m) {
@@ -477,6 +499,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
 struct EncodeTcArgs {
     const __nv_bfloat16 *Q;   // [H,M,D] (read directly in the head-pair form)
+    const float *lse_dec;     // [B,N,H]: only for the backward's dZ form of the kernel
     const uint8_t *key_mask;  // [B,N] or null
     float *part_m, *part_l, *part_acc;
     uint32_t *status;
@@ -495,8 +518,10 @@ struct EncodeSmem {
     static constexpr size_t kv_off = 0;                         // [stage][K tile | V tile]
     __host__ __device__ static size_t q_off() { return (size_t)kEncStages * 2 * G::TILE_BYTES; }
     __host__ __device__ static size_t bar_off() { return q_off() + (size_t)2 * kTile * G::RB; }
+    static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 32 * sizeof(float);   // per softmax warp: 2 x 32 column addends
+    __host__ __device__ static size_t col_off() { return bar_off() + 512; }
     __host__ __device__ static size_t total() {
-        size_t t = bar_off() + 512 + 1024;
+        size_t t = col_off() + kColBytes + 1024;
         return t < kTcMinSmem ? kTcMinSmem : t;
     }
 };
@@ -515,7 +540,12 @@ struct EncodeSmem {
 // 2p+1; the A operand is the block-diagonal [Q_2p 0; 0 Q_2p+1] over the 2D feature columns the two heads occupy
 // side by side in a token row, so one MMA with K = 2D gives every lane its own head's scores, and the value MMA
 // with N = 2D gives lanes 0-63 their rows in accumulator columns [0, D) and lanes 64-127 theirs in [D, 2D).
-template <int D, bool kPair>
+//
+// dZ form (kDz; pass A of the backward): the same kernel with dY in place of V and the decode weights in place of
+// the encode weights, dZ_m = sum_n exp(S[m,n] - lse_dec[n]) dY_n.  Every column (token) carries its own shift
+// and the weights are already normalised, so there is no running maximum, no rescaling and no sum; tokens
+// beyond N get the shift -inf.  Every group leaves one partial sum of dZ per split (part_acc).
+template <int D, bool kPair, bool kDz = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
@@ -646,8 +676,11 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const uint64_t vdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES),
                                                       G::SBO, G::SBO, G::SWZ) + (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
 #pragma unroll
-                for (int k = 0; k < UNIT / 16; ++k)
+                for (int k = 0; k < UNIT / 16; ++k) {
                     ptx::mma_ts(dcol, gcol + w * UNIT + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, (n > 0 || k > 0) ? 1u : 0u);
+                    if (kDz)    // the lo halves of the weights sit 16 columns further on
+                        ptx::mma_ts(dcol, gcol + w * UNIT + 16 + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, 1u);
+                }
                 ptx::mma_commit(bar(PV_DONE + g));
                 if (w == 1) {                                               // the tile's last unit: one arrival per group
                     ptx::mma_commit(bar(KV_EMPTY + s));
@@ -669,6 +702,29 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         float2 l2 = make_float2(0.f, 0.f);
         int done = 0;                                           // units finished
         bool ok = true;
+        float *colneg = reinterpret_cast<float *>(smem + SM::col_off()) + (warp - kFirstSoftmaxWarp) * 64;   // this warp's addends
+        // dZ form of a unit: weights exp(S - lse_dec[token]), no maximum, no sum.
+        auto unit_dz = [&](int t, int w) -> bool {
+            const uint32_t sbase = gcol + w * UNIT;
+            const int n = t * kTile + c * HALF + w * UNIT + lane;          // this lane fetches the shift of token n
+            const int hh = h + (kPair ? (row >> 6) : 0);                   // the head of this lane's latent
+            __syncwarp();                                                   // the previous unit's reads are done
+            colneg[lane] = n < a.N ? -a.lse_dec[((size_t)b * a.N + n) * a.H + hh] * 1.4426950408889634f : -INFINITY;
+            __syncwarp();
+            if (!warp_wait(bar(S_FULL + 2 * g + w), (done >> 1) & 1, abort_flag, kErrEncode | 5)) return false;
+            ptx::tc_fence_after();
+            uint32_t r[32], pk[16], pl[16];
+            ptx::tmem_ld32(sbase, r);
+            ptx::tmem_wait_ld();
+            exp_chunk_cols<32>(r, pk, pl, sl2p, colneg);
+            ptx::tmem_st16(sbase, pk);                          // hi halves over the first 16 score columns,
+            ptx::tmem_st16(sbase + 16, pl);                     // lo halves over the other 16
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(bar(P_FULL + 2 * g + w));
+            ++done;
+            return true;
+        };
         // One unit of work: 32 token columns of this group's half, on score buffer w.  kMasked: some of the tile's
         // tokens may be padding or lie beyond N (their weights are exactly 0); the plain form has no such tests.
         auto unit = [&](auto masked, int t, int w) -> bool {
@@ -730,7 +786,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;   // warp-uniform
 #pragma unroll 1
                 for (int w = 0; ok && w < 2; ++w)               // the half's two units, on alternating buffers
-                    ok = plain ? unit(std::false_type{}, t, w) : unit(std::true_type{}, t, w);
+                    ok = kDz ? unit_dz(t, w) : plain ? unit(std::false_type{}, t, w) : unit(std::true_type{}, t, w);
             }
         }
         // write this group's partial (running max in natural-log units, sum, un-normalised rows)
@@ -754,8 +810,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const long rows = (long)a.B * a.H * M;
             const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);
             const size_t prow = (size_t)part * rows + ((size_t)b * a.H + h + second) * M + m;
-            a.part_m[prow] = (m_run == -INFINITY) ? -INFINITY : m_run * a.scale;
-            a.part_l[prow] = l2.x + l2.y;
+            if (!kDz) {
+                a.part_m[prow] = (m_run == -INFINITY) ? -INFINITY : m_run * a.scale;
+                a.part_l[prow] = l2.x + l2.y;
+            }
             float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * D);
 #pragma unroll
             for (int dc = 0; dc < D / 4; ++dc)
