@@ -11,6 +11,7 @@
 #include "flare_simt.cuh"
 #include "flare_bwd.cuh"
 #include "flare_tc.cuh"
+#include "flare_bwd_tc.cuh"
 
 using namespace flare;
 
@@ -229,6 +230,34 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
 }
 
 template <int D>
+int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
+                     const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
+                     const float *lse_dec, const float *dd, float *part, uint32_t *status, cudaStream_t st) {
+    CUtensorMap tmK, tmV, tmG, tmQ;
+    int rc;
+    if ((rc = make_token_map(&tmK, K, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmV, V, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmG, dY, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
+    const size_t smem = BwdDqSmem<D>::total();
+    static bool attr_set = false;
+    if (!attr_set) {
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    BwdDqTcArgs a;
+    a.Z = Z; a.dZ = dZ; a.lse_enc = lse_enc; a.de = de; a.lse_dec = lse_dec; a.dd = dd;
+    a.key_mask = mask; a.part = part; a.status = status;
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.sl2 = d->scale * kLog2e;
+    a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
+    dim3 grid(p.splits, d->H * p.pairs, d->B);
+    bwd_dq_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+template <int D>
 int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
                      float *lse_dec, uint32_t *status, cudaStream_t st) {
     CUtensorMap tmK, tmQ;
@@ -298,6 +327,25 @@ int launch_decode_simt(const flare_desc_t *d, const void *Q, const void *K, cons
 // Pass A (dZ) runs as the dZ form of the tensor-core encode kernel wherever that kernel runs.
 bool bwd_dz_on_tensor_cores(const flare_desc_t *d) { return use_tc(d); }
 
+// Pass B for dQ runs on the tensor cores for narrow heads (S, A, C and the partial dQ of a group share its 128
+// TMEM columns: 3 * 32 + D).
+bool bwd_dq_on_tensor_cores(const flare_desc_t *d) { return use_tc(d) && d->D <= 32; }
+
+// Plan of the tensor-core dQ kernel: the encode plan without head pairing.
+TcEncodePlan tc_dq_plan(const flare_desc_t *d, int sms) {
+    TcEncodePlan p;
+    const int mb = (d->M + kTile - 1) / kTile;
+    p.tiles = (d->N + kTile - 1) / kTile;
+    p.pairs = (mb + 1) / 2;
+    long s = sms / ((long)d->B * d->H * p.pairs);
+    if (s < 1) s = 1;
+    if (s > p.tiles) s = p.tiles;
+    p.splits = (int)s;
+    p.per_split = (mb == 1) ? 4 : 2;
+    p.P = p.splits * p.per_split;
+    return p;
+}
+
 SimtPlan bwd_dq_plan(const flare_desc_t *d, int sms) {
     SimtPlan p = simt_plan(d, sms);
     if (p.LM > 64) p.LM = 64;
@@ -317,6 +365,7 @@ BwdLayout bwd_layout(const flare_desc_t *d, int sms) {
     const int pa = simt_plan(d, sms).P, pb = bwd_dq_plan(d, sms).P;
     w.P = pa > pb ? pa : pb;
     if (bwd_dz_on_tensor_cores(d) && tc_encode_plan(d, sms).P > w.P) w.P = tc_encode_plan(d, sms).P;
+    if (bwd_dq_on_tensor_cores(d) && tc_dq_plan(d, sms).P > w.P) w.P = tc_dq_plan(d, sms).P;
     size_t off = kHeaderBytes;
     w.part = off; off += align_up(sizeof(float) * (size_t)w.P * rows * d->D);
     w.dz = off;   off += align_up(sizeof(float) * (size_t)rows * d->D);
@@ -371,19 +420,32 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
         (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, lse_enc, lse_dec, (T *)dK, (T *)dV, dd,
         d->B, d->H, d->N, d->M, d->scale);
     FLARE_CUDA(cudaGetLastError());
-    const size_t dyn = sizeof(float) * 3 * (size_t)pb.LM * (D + 1);
-    static bool attr_set = false;
-    if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)(sizeof(float) * 3 * 64 * (D + 1))));
-        attr_set = true;
+    int dq_parts = pb.P;
+    bool dq_on_tc = false;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && (D == 16 || D == 32)) {
+        if (bwd_dq_on_tensor_cores(d)) {
+            const int rc = launch_bwd_dq_tc<D>(d, tc_dq_plan(d, sms), Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part,
+                                               reinterpret_cast<uint32_t *>(ws), st);
+            if (rc != FLARE_OK) return rc;
+            dq_parts = tc_dq_plan(d, sms).P;
+            dq_on_tc = true;
+        }
     }
-    bwd_dq_simt_kernel<T, D><<<dim3(pb.splits, d->H, d->B), kBwdThreads, dyn, st>>>(
-        (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, dd, lse_enc, lse_dec, part, d->B, d->H,
-        d->N, d->M, pb.LM, pb.chunk, d->scale);
-    FLARE_CUDA(cudaGetLastError());
+    if (!dq_on_tc) {
+        const size_t dyn = sizeof(float) * 3 * (size_t)pb.LM * (D + 1);
+        static bool attr_set = false;
+        if (!attr_set) {
+            FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)(sizeof(float) * 3 * 64 * (D + 1))));
+            attr_set = true;
+        }
+        bwd_dq_simt_kernel<T, D><<<dim3(pb.splits, d->H, d->B), kBwdThreads, dyn, st>>>(
+            (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, dd, lse_enc, lse_dec, part, d->B, d->H,
+            d->N, d->M, pb.LM, pb.chunk, d->scale);
+        FLARE_CUDA(cudaGetLastError());
+    }
     const long per_batch = (long)d->H * d->M * d->D;
-    bwd_dq_reduce_kernel<<<(unsigned)((per_batch + 255) / 256), 256, 0, st>>>(part, dQ, pb.P, d->B, d->H, d->M, d->D,
+    bwd_dq_reduce_kernel<<<(unsigned)((per_batch + 255) / 256), 256, 0, st>>>(part, dQ, dq_parts, d->B, d->H, d->M, d->D,
                                                                              d->scale);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
