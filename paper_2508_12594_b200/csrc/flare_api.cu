@@ -258,6 +258,38 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
 }
 
 template <int D>
+int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
+                        const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
+                        const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st) {
+    CUtensorMap tmK, tmV, tmG, tmQ;
+    int rc;
+    if ((rc = make_token_map(&tmK, K, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmV, V, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_token_map(&tmG, dY, d, kTile)) != FLARE_OK) return rc;
+    if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
+    BwdTokTcArgs a;
+    a.stages = BwdTokSmem<D>::stages(d->M);
+    if (a.stages < 1) return FLARE_ERR_UNSUPPORTED;
+    const size_t smem = BwdTokSmem<D>::total(a.stages, d->M);
+    static bool attr_set = false;
+    if (!attr_set) {
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    a.Z = Z; a.dZ = dZ; a.lse_enc = lse_enc; a.de = de; a.lse_dec = lse_dec; a.key_mask = mask;
+    a.dK = (__nv_bfloat16 *)dK; a.dV = (__nv_bfloat16 *)dV; a.dd = dd; a.status = status;
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.scale = d->scale; a.sl2 = d->scale * kLog2e;
+    a.tiles = (d->N + kTile - 1) / kTile;
+    long per_head = sms / ((long)d->B * d->H);
+    if (per_head < 1) per_head = 1;
+    if (per_head > a.tiles) per_head = a.tiles;
+    bwd_token_tc_kernel<D><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+template <int D>
 int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
                      float *lse_dec, uint32_t *status, cudaStream_t st) {
     CUtensorMap tmK, tmQ;
@@ -416,10 +448,21 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     FLARE_CUDA(cudaGetLastError());
     bwd_de_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(dZ, Z, de, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
-    bwd_token_simt_kernel<T, D><<<dim3((d->N + 127) / 128, d->H, d->B), 128, 0, st>>>(
-        (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, lse_enc, lse_dec, (T *)dK, (T *)dV, dd,
-        d->B, d->H, d->N, d->M, d->scale);
-    FLARE_CUDA(cudaGetLastError());
+    bool tok_on_tc = false;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && (D == 16 || D == 32)) {
+        if (bwd_dq_on_tensor_cores(d) && BwdTokSmem<D>::stages(d->M) >= 1) {
+            const int rc = launch_bwd_token_tc<D>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd,
+                                                  reinterpret_cast<uint32_t *>(ws), st);
+            if (rc != FLARE_OK) return rc;
+            tok_on_tc = true;
+        }
+    }
+    if (!tok_on_tc) {
+        bwd_token_simt_kernel<T, D><<<dim3((d->N + 127) / 128, d->H, d->B), 128, 0, st>>>(
+            (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, lse_enc, lse_dec, (T *)dK, (T *)dV, dd,
+            d->B, d->H, d->N, d->M, d->scale);
+        FLARE_CUDA(cudaGetLastError());
+    }
     int dq_parts = pb.P;
     bool dq_on_tc = false;
     if constexpr (std::is_same<T, __nv_bfloat16>::value && (D == 16 || D == 32)) {

@@ -304,4 +304,340 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
 }
 
+// ------------------------------------------------------------------------------- pass B, token side (dK, dV)
+// Tokens on the 128 TMEM lanes, latents on columns in units of kUnit, every softmax group a token tile of its
+// own.  Two sweeps over the latents of a tile, as in the CUDA-core kernel: the first needs S^T = K Q^T and
+// A^T = dY Z^T and leaves dd[n] = sum_m W_dec[n,m] A[n,m] in a register; the second adds C^T = V dZ^T, turns the
+// three into dS^T and W_enc^T (two bf16 halves each) over the columns just read, and two more contractions
+// accumulate dK_n = scale * sum_m dS[m,n] q_m and dV_n = sum_m W_enc[m,n] dZ_m.  dd goes to the workspace for
+// the dQ kernel.  Columns of a group: S, A, C (kUnit each), dK (D), dV (D): 3 kUnit + 2 D <= 128.
+template <int D>
+struct BwdTokGeom {
+    static constexpr int kUnit = D == 16 ? 32 : 16;
+    static constexpr int kMaxStages = 8;
+};
+
+struct BwdTokTcArgs {
+    const float *Z, *dZ;       // [B,H,M,D]
+    const float *lse_enc, *de; // [B,H,M]
+    const float *lse_dec;      // [B,N,H]
+    const uint8_t *key_mask;   // [B,N] or null
+    __nv_bfloat16 *dK, *dV;    // [B,N,H,D]
+    float *dd;                 // [B,N,H] out
+    uint32_t *status;
+    int B, H, N, M;
+    float scale, sl2;
+    int tiles, stages;
+};
+
+template <int D>
+struct BwdTokSmem {
+    using G = TileGeom<D>;
+    __host__ __device__ static int padded_m(int M) { return (M + 31) & ~31; }
+    // tiles: [stage][K | V | dY]; latents: Q, Z_hi, Z_lo, dZ_hi, dZ_lo with padded_m rows each; then -lse_enc, -de
+    __host__ __device__ static size_t lat_off(int stages, int M, int which) {
+        return (size_t)stages * 3 * G::TILE_BYTES + (size_t)which * padded_m(M) * G::RB;
+    }
+    __host__ __device__ static size_t cst_off(int stages, int M) { return lat_off(stages, M, 5); }
+    __host__ __device__ static size_t bar_off(int stages, int M) { return cst_off(stages, M) + 2 * sizeof(float) * padded_m(M); }
+    __host__ __device__ static size_t total(int stages, int M) {
+        size_t t = bar_off(stages, M) + 512 + 1024;
+        return t < kTcMinSmem ? kTcMinSmem : t;
+    }
+    // the most stages (at most kMaxStages) that fit beside the latent operands; 0 if not even one does
+    __host__ static int stages(int M) {
+        int s = BwdTokGeom<D>::kMaxStages;
+        while (s > 0 && total(s, M) > (size_t)227 * 1024) --s;
+        return s;
+    }
+};
+
+// grid = (CTAs per head, H, B); a CTA takes the token tiles blockIdx.x, blockIdx.x + gridDim.x, ...
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, 1)
+bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                    const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdTokTcArgs a) {
+    using G = TileGeom<D>;
+    using SM = BwdTokSmem<D>;
+    constexpr int UNIT = BwdTokGeom<D>::kUnit;
+    constexpr int kMaxSt = BwdTokGeom<D>::kMaxStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int M = a.M, MU = SM::padded_m(M), stages = a.stages;
+    uint8_t *sQ = smem + SM::lat_off(stages, M, 0);
+    float *cst = reinterpret_cast<float *>(smem + SM::cst_off(stages, M));      // [MU] -lse_enc (log2 units), [MU] -de
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off(stages, M));
+    constexpr int NG = kSoftmaxGroups;
+    enum { T_FULL = 0, T_EMPTY = T_FULL + kMaxSt, S_FULL = T_EMPTY + kMaxSt, P_FULL = S_FULL + NG,
+           ACC_FULL = P_FULL + NG, ACC_FREE = ACC_FULL + NG, Q_FULL = ACC_FREE + NG, NBARS };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int nt = (a.tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // tiles of this CTA
+    const int ng = stages < NG ? stages : NG;                   // groups at work
+    const int nu = (M + UNIT - 1) / UNIT;                       // latent units per sweep
+    constexpr uint32_t NCOLS = 512;
+    auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NBARS; ++i)
+            ptx::mbar_init(bar(i), ((i >= P_FULL && i < P_FULL + NG) || (i >= ACC_FREE && i < ACC_FREE + NG)) ? 128u : 1u);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmK);
+        ptx::prefetch_tensormap(&tmV);
+        ptx::prefetch_tensormap(&tmG);
+        ptx::prefetch_tensormap(&tmQ);
+    }
+    if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), NCOLS);
+    // latent rows M..MU-1 of all five operands are zero; their columns carry -lse_enc = -inf
+    for (int i = threadIdx.x; i < 5 * (MU - M) * (G::RB / 16); i += kTcThreads) {
+        const int which = i / ((MU - M) * (G::RB / 16)), rem = i % ((MU - M) * (G::RB / 16));
+        reinterpret_cast<uint4 *>(smem + SM::lat_off(stages, M, which) + (size_t)M * G::RB)[rem] = make_uint4(0, 0, 0, 0);
+    }
+    for (int m = threadIdx.x; m < MU; m += kTcThreads) {
+        float nle = -INFINITY, nde = 0.f;
+        if (m < M) {
+            const size_t r = ((size_t)b * a.H + h) * M + m;
+            const float le = a.lse_enc[r];
+            nle = (le == -INFINITY) ? -INFINITY : -le * 1.4426950408889634f;
+            nde = -a.de[r];
+        }
+        cst[m] = nle;
+        cst[MU + m] = nde;
+    }
+    for (int i = threadIdx.x; i < 2 * M * (D / 8); i += kTcThreads) {
+        const int which = i / (M * (D / 8)), rem = i % (M * (D / 8)), m = rem / (D / 8), ch = rem % (D / 8);
+        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + m) * D + ch * 8;
+        const float4 lo4 = *reinterpret_cast<const float4 *>(src), hi4 = *reinterpret_cast<const float4 *>(src + 4);
+        const float z[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+        uint32_t vh[4], vl[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            vh[k] = ptx::pack_bf16(z[2 * k], z[2 * k + 1]);
+            vl[k] = ptx::pack_bf16(z[2 * k] - __uint_as_float(vh[k] << 16), z[2 * k + 1] - __uint_as_float(vh[k] & 0xffff0000u));
+        }
+        const size_t off = (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4);
+        *reinterpret_cast<uint4 *>(smem + SM::lat_off(stages, M, 1 + 2 * which) + off) = make_uint4(vh[0], vh[1], vh[2], vh[3]);
+        *reinterpret_cast<uint4 *>(smem + SM::lat_off(stages, M, 2 + 2 * which) + off) = make_uint4(vl[0], vl[1], vl[2], vl[3]);
+    }
+    ptx::fence_proxy_async_smem();
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tm = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
+            for (int r = 0; r < M; r += 16)
+                ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+            for (int i = 0; i < nt; ++i) {
+                const int s = i % stages, t = blockIdx.x + i * gridDim.x;
+                if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / stages) & 1) ^ 1, abort_flag, kErrBwdTok | 1)) break;
+                ptx::mbar_arrive_expect_tx(bar(T_FULL + s), 3 * G::TILE_BYTES);
+                uint8_t *dst = smem + (size_t)s * 3 * G::TILE_BYTES;
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * D, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * D, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * D, t * kTile, b);
+            }
+        }
+    } else if (warp < kFirstSoftmaxWarp) {
+        const int g = warp - kFirstIssuerWarp;
+        if (lane == 0 && g < ng) {
+            const uint32_t idescS = ptx::instr_desc_bf16(128, UNIT, 0, 0);
+            const uint32_t idescO = ptx::instr_desc_bf16(128, D, 0, 1);
+            const uint32_t gcol = tm + g * 128;
+            const uint32_t kcol = gcol + 3 * UNIT, vcol = kcol + D;       // the dK and dV accumulators
+            bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrBwdTok | 2);
+            uint32_t cnt = 0;
+            int k_tile = 0;
+            for (int i = g; ok && i < nt; i += ng, ++k_tile) {
+                const int s = i % stages;
+                if (!ptx::mbar_wait(bar(T_FULL + s), (i / stages) & 1, abort_flag, kErrBwdTok | 3)) break;
+                ptx::tc_fence_after();
+                const uint32_t tbase = ptx::smem_u32(smem + (size_t)s * 3 * G::TILE_BYTES);
+                // the tile's token rows as the K-major A operand of the three score-like contractions
+                const uint64_t kdesc = ptx::smem_desc(tbase, 16, G::SBO, G::SWZ);
+                const uint64_t vdesc = ptx::smem_desc(tbase + G::TILE_BYTES, 16, G::SBO, G::SWZ);
+                const uint64_t gdesc = ptx::smem_desc(tbase + 2 * G::TILE_BYTES, 16, G::SBO, G::SWZ);
+                for (int sweep = 0; ok && sweep < 2; ++sweep) {
+                    for (int u = 0; u < nu; ++u) {
+                        const uint64_t uoff = (uint64_t)(u * UNIT * G::RB / 16);      // the unit's latent rows
+                        uint64_t ld[5];
+#pragma unroll
+                        for (int w = 0; w < 5; ++w)
+                            ld[w] = ptx::smem_desc(ptx::smem_u32(smem + SM::lat_off(stages, M, w)), 16, G::SBO, G::SWZ) + uoff;
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol, kdesc + 2 * k, ld[0] + 2 * k, idescS, k > 0);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + UNIT, gdesc + 2 * k, ld[1] + 2 * k, idescS, k > 0);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + UNIT, gdesc + 2 * k, ld[2] + 2 * k, idescS, 1u);
+                        if (sweep == 1) {
+#pragma unroll
+                            for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + 2 * UNIT, vdesc + 2 * k, ld[3] + 2 * k, idescS, k > 0);
+#pragma unroll
+                            for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + 2 * UNIT, vdesc + 2 * k, ld[4] + 2 * k, idescS, 1u);
+                        }
+                        ptx::mma_commit(bar(S_FULL + g));
+                        if (!ptx::mbar_wait(bar(P_FULL + g), cnt & 1, abort_flag, kErrBwdTok | 4)) { ok = false; break; }
+                        ++cnt;
+                        ptx::tc_fence_after();
+                        if (sweep == 1) {
+                            // the previous tile's accumulators must have been read before they are overwritten
+                            if (u == 0 && k_tile > 0 &&
+                                !ptx::mbar_wait(bar(ACC_FREE + g), (k_tile - 1) & 1, abort_flag, kErrBwdTok | 5)) { ok = false; break; }
+                            ptx::tc_fence_after();
+                            // Q and dZ (hi, lo) rows of the unit as MN-major B operands, 16 latent rows per k-step
+                            const uint64_t qmn = ptx::smem_desc(ptx::smem_u32(smem + SM::lat_off(stages, M, 0)), G::SBO, G::SBO, G::SWZ) + uoff;
+                            const uint64_t zmn = ptx::smem_desc(ptx::smem_u32(smem + SM::lat_off(stages, M, 3)), G::SBO, G::SBO, G::SWZ) + uoff;
+                            const uint64_t zln = ptx::smem_desc(ptx::smem_u32(smem + SM::lat_off(stages, M, 4)), G::SBO, G::SBO, G::SWZ) + uoff;
+#pragma unroll
+                            for (int k = 0; k < UNIT / 16; ++k) {
+                                const uint32_t acc = (u > 0 || k > 0) ? 1u : 0u;
+                                ptx::mma_ts(kcol, gcol + k * 8, qmn + (uint64_t)(k * G::RB), idescO, acc);              // dS hi
+                                ptx::mma_ts(kcol, gcol + UNIT + k * 8, qmn + (uint64_t)(k * G::RB), idescO, 1u);        // dS lo
+                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 8, zmn + (uint64_t)(k * G::RB), idescO, acc);   // W_enc dZ_hi
+                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 8, zln + (uint64_t)(k * G::RB), idescO, 1u);    // W_enc dZ_lo
+                                ptx::mma_ts(vcol, gcol + UNIT / 2 + k * 8, zmn + (uint64_t)(k * G::RB), idescO, 1u);    // W_enc lo x dZ_hi
+                            }
+                        }
+                    }
+                }
+                if (!ok) break;
+                ptx::mma_commit(bar(T_EMPTY + s));
+                ptx::mma_commit(bar(ACC_FULL + g));
+            }
+        }
+    } else {
+        const int g = (warp - kFirstSoftmaxWarp) >> 2;
+        const int row = ((warp & 3) << 5) + lane;               // TMEM lane = token within the tile
+        const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
+        const uint32_t gcol = tm + lane_addr + g * 128;
+        const uint32_t kcol = gcol + 3 * UNIT, vcol = kcol + D;
+        const float2 sl2p = make_float2(a.sl2, a.sl2);
+        uint32_t cnt = 0;
+        int k_tile = 0;
+        bool ok = true;
+        for (int i = g; ok && g < ng && i < nt; i += ng, ++k_tile) {
+            const int t = blockIdx.x + i * gridDim.x, n = t * kTile + row;
+            const bool inside = n < a.N;
+            const bool valid = inside && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0);
+            const size_t tok = ((size_t)b * a.N + (inside ? n : 0)) * a.H + h;
+            const float negld = inside ? -a.lse_dec[tok] * 1.4426950408889634f : -INFINITY;
+            const float2 negldp = make_float2(negld, negld);
+            const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;      // uniform over the group
+            // sweep 1: dd[n] = sum_m W_dec[n,m] (dY_n . Z_m)
+            float2 dd2 = make_float2(0.f, 0.f);
+            for (int u = 0; ok && u < nu; ++u) {
+                if (!warp_wait(bar(S_FULL + g), cnt & 1, abort_flag, kErrBwdTok | 6)) { ok = false; break; }
+                ++cnt;
+                ptx::tc_fence_after();
+#pragma unroll
+                for (int hb = 0; hb < UNIT / 16; ++hb) {
+                    uint32_t s[16], av[16];
+                    ptx::tmem_ld16(gcol + hb * 16, s);
+                    ptx::tmem_ld16(gcol + UNIT + hb * 16, av);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * k]), __uint_as_float(s[2 * k + 1])), sl2p, negldp);
+                        dd2 = __ffma2_rn(make_float2(ptx::ex2(x.x), ptx::ex2(x.y)),
+                                         make_float2(__uint_as_float(av[2 * k]), __uint_as_float(av[2 * k + 1])), dd2);
+                    }
+                }
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(bar(P_FULL + g));
+            }
+            const float dd = dd2.x + dd2.y;
+            const float2 negddp = make_float2(-dd, -dd);
+            // sweep 2: dS^T and W_enc^T of every unit, handed to the issuing warp
+            auto unit2 = [&](auto masked, int u) {
+                constexpr bool kMasked = decltype(masked)::value;
+                uint32_t pwl[UNIT / 2];                                             // lo halves of W_enc, stored last
+#pragma unroll
+                for (int qd = 0; qd < UNIT / 8; ++qd) {
+                    uint32_t s[8], av[8], cv[8], pk[4], pl[4], pw[4];
+                    ptx::tmem_ld8(gcol + qd * 8, s);
+                    ptx::tmem_ld8(gcol + UNIT + qd * 8, av);
+                    ptx::tmem_ld8(gcol + 2 * UNIT + qd * 8, cv);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int col = u * UNIT + qd * 8 + 2 * k;                  // latent of this pair of columns
+                        const float2 sp = make_float2(__uint_as_float(s[2 * k]), __uint_as_float(s[2 * k + 1]));
+                        const float2 nle = *reinterpret_cast<const float2 *>(cst + col);
+                        const float2 nde = *reinterpret_cast<const float2 *>(cst + MU + col);
+                        const float2 xd = __ffma2_rn(sp, sl2p, negldp), xe = __ffma2_rn(sp, sl2p, nle);
+                        const float2 pd = make_float2(ptx::ex2(xd.x), ptx::ex2(xd.y));
+                        float2 pe = make_float2(ptx::ex2(xe.x), ptx::ex2(xe.y));
+                        if (kMasked && !valid) pe = make_float2(0.f, 0.f);
+                        const float2 uu = __fadd2_rn(make_float2(__uint_as_float(av[2 * k]), __uint_as_float(av[2 * k + 1])), negddp);
+                        const float2 vv = __fadd2_rn(make_float2(__uint_as_float(cv[2 * k]), __uint_as_float(cv[2 * k + 1])), nde);
+                        const float2 ds = __ffma2_rn(pd, uu, __fmul2_rn(pe, vv));
+                        const uint32_t hi = ptx::pack_bf16(ds.x, ds.y);
+                        pk[k] = hi;
+                        pl[k] = ptx::pack_bf16(ds.x - __uint_as_float(hi << 16), ds.y - __uint_as_float(hi & 0xffff0000u));
+                        const uint32_t wh = ptx::pack_bf16(pe.x, pe.y);
+                        pw[k] = wh;
+                        pwl[qd * 4 + k] = ptx::pack_bf16(pe.x - __uint_as_float(wh << 16), pe.y - __uint_as_float(wh & 0xffff0000u));
+                    }
+                    // packed results over columns this thread has already read: dS hi over S, dS lo over A, W_enc over C
+                    ptx::tmem_st4(gcol + qd * 4, pk);
+                    ptx::tmem_st4(gcol + UNIT + qd * 4, pl);
+                    ptx::tmem_st4(gcol + 2 * UNIT + qd * 4, pw);
+                }
+                // the upper half of the score columns is free once all of them have been read
+                if (UNIT == 32) ptx::tmem_st16(gcol + UNIT / 2, pwl); else ptx::tmem_st8(gcol + UNIT / 2, pwl);
+            };
+            for (int u = 0; ok && u < nu; ++u) {
+                if (!warp_wait(bar(S_FULL + g), cnt & 1, abort_flag, kErrBwdTok | 7)) { ok = false; break; }
+                ++cnt;
+                ptx::tc_fence_after();
+                if (plain) unit2(std::false_type{}, u); else unit2(std::true_type{}, u);
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(bar(P_FULL + g));
+            }
+            if (!ok) break;
+            if (!warp_wait(bar(ACC_FULL + g), k_tile & 1, abort_flag, kErrBwdTok | 8)) { ok = false; break; }
+            ptx::tc_fence_after();
+            uint32_t ak[D], avv[D];
+#pragma unroll
+            for (int dc = 0; dc < D / 16; ++dc) {
+                ptx::tmem_ld16(kcol + dc * 16, ak + dc * 16);
+                ptx::tmem_ld16(vcol + dc * 16, avv + dc * 16);
+            }
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(bar(ACC_FREE + g));
+            if (inside) {
+                a.dd[tok] = dd;
+                uint4 *dk = reinterpret_cast<uint4 *>(a.dK + tok * D), *dv = reinterpret_cast<uint4 *>(a.dV + tok * D);
+#pragma unroll
+                for (int q = 0; q < D / 8; ++q) {
+                    uint32_t wk[4], wv4[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        wk[k] = ptx::pack_bf16(__uint_as_float(ak[8 * q + 2 * k]) * a.scale, __uint_as_float(ak[8 * q + 2 * k + 1]) * a.scale);
+                        wv4[k] = ptx::pack_bf16(__uint_as_float(avv[8 * q + 2 * k]), __uint_as_float(avv[8 * q + 2 * k + 1]));
+                    }
+                    dk[q] = make_uint4(wk[0], wk[1], wk[2], wk[3]);
+                    dv[q] = make_uint4(wv4[0], wv4[1], wv4[2], wv4[3]);
+                }
+            }
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == kFirstIssuerWarp) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tm, NCOLS);
+    }
+    if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
+}
+
 }  // namespace flare

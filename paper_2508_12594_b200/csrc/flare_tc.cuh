@@ -38,7 +38,7 @@ constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode)
 constexpr size_t kTcMinSmem = 120 * 1024;  // request at least this much so that one CTA owns an SM (and its TMEM)
 
 // Error codes left in the workspace header by a wait that gave up.
-enum : uint32_t { kErrDecode = 0x100, kErrEncode = 0x200, kErrBwdDq = 0x300 };
+enum : uint32_t { kErrDecode = 0x100, kErrEncode = 0x200, kErrBwdDq = 0x300, kErrBwdTok = 0x400 };
 
 // Bounded wait whose outcome is the same for every lane of the warp, so that the warp-collective tensor-memory
 // instructions that follow are executed by all lanes or by none.
