@@ -152,6 +152,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override N (a smaller case of the same workload)")
+    ap.add_argument("--no-backward", action="store_true", help="skip the forward+backward leg")
     args = ap.parse_args()
     w = get_workload(args.workload)
     if args.tokens > 0:
@@ -233,6 +234,40 @@ def main():
             a.record(stream); fn(); b.record(stream)
         torch.cuda.synchronize()
         stage_ms[name] = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)
+    # forward + backward of the same batch (reported beside the forward-only metric): dY is seeded noise
+    fwd_bwd = None
+    if not args.no_backward:
+        gen = torch.Generator(device="cuda").manual_seed(wr.seed + 7)
+        dYt = torch.randn(K.shape, generator=gen, device="cuda", dtype=torch.float32).to(K.dtype)
+        le = torch.empty(w.B, w.H, w.M, dtype=torch.float32, device="cuda")
+        ld = torch.empty(w.B, w.N, w.H, dtype=torch.float32, device="cuda")
+        wsb = flare.alloc_workspace(desc, flare.OP_BACKWARD)
+        dQ = torch.empty(w.H, w.M, w.D, dtype=torch.float32, device="cuda")
+        dK, dV = torch.empty_like(K), torch.empty_like(V)
+
+        def both():
+            if flush is not None:
+                flush.zero_()
+            flare.flare_forward(desc, Q, K, V, mask, Y, Z, le, ld, ws, stream)
+            flare.flare_backward(desc, Q, K, V, mask, Y, dYt, Z, le, ld, dQ, dK, dV, wsb, stream)
+
+        nb = max(1, min(args.steps, 50))
+        for _ in range(3):
+            both()
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nb)]
+        for a, b in pairs:
+            if flush is not None:
+                flush.zero_()
+            a.record(stream)
+            flare.flare_forward(desc, Q, K, V, mask, Y, Z, le, ld, ws, stream)
+            flare.flare_backward(desc, Q, K, V, mask, Y, dYt, Z, le, ld, dQ, dK, dV, wsb, stream)
+            b.record(stream)
+        torch.cuda.synchronize()
+        flare.flare_check(wsb)
+        fb_ms = sum(a.elapsed_time(b) for a, b in pairs) / nb
+        fwd_bwd = {"ms_per_step": fb_ms, "value": w.tokens / (fb_ms / 1e3), "unit": "tokens/s", "steps": nb,
+                   "gpu_launches_per_step": 10, "note": "per GPU; forward with saved statistics, then backward"}
+        del dYt, dK, dV, wsb
     clocks = sampler.stop() if rank == 0 else None
     flare.flare_check(ws)
 
@@ -250,7 +285,7 @@ def main():
         if dist is not None:
             dist.destroy_process_group()
         return
-    finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist)
+    finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist, fwd_bwd)
 
 
 def run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V, mask, tensor_bytes, e):
@@ -278,7 +313,7 @@ def run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V
             "d2h_bytes_per_step": tensor_bytes, "ms_per_step": e2e_ms}
 
 
-def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist):
+def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist, fwd_bwd=None):
     peaks, peak_kind = load_peaks()
     # Roofline of the slower main kernel.  Per stage and head the contraction work is 4*N*M*D FLOP (scores and
     # value contraction); the bytes are K and V read (encode) or K read and Y written (decode), plus Q_lat.
@@ -313,6 +348,8 @@ def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_by
                    "l2": l2_note, "parallelism": f"replicas x{world}"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roof,
     }
+    if fwd_bwd is not None:
+        out["fwd_bwd"] = fwd_bwd
     if not args.no_cpu_baseline:
         v, dt, n, cores = oracle_sample(w, inp, args.cpu_tokens)
         out["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",

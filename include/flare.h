@@ -117,6 +117,8 @@ int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, co
  * Z, lse_enc, lse_dec are the ones flare_forward wrote; Y is its output (part of the saved set; the present
  * kernels rebuild dY_n.Y_n = sum_m W_dec[n,m] (dY_n.Z_m) in float32 instead of reading the rounded Y, which
  * is markedly more accurate where the latent rows a token mixes are nearly equal).
+ * bfloat16 inputs run all three passes (dZ; dK, dV; dQ_lat) on the tensor cores (the last two for D <= 32), with
+ * every rounded factor of a cancelling sum carried as two bfloat16 halves; float32 inputs run on the CUDA cores.
  * dQ_lat, dK, dV are overwritten.  Workspace: flare_workspace_bytes(desc, FLARE_OP_BACKWARD) bytes holding dZ,
  * per-split partial sums of dZ and dQ_lat, and one float per (b, n, h); nothing of size N x M.
  */

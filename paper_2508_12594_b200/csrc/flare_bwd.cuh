@@ -1,4 +1,7 @@
-// Backward of the FLARE mixer on the CUDA cores (float32 arithmetic, any supported dtype and shape).
+// Backward of the FLARE mixer on the CUDA cores (float32 arithmetic, any supported dtype and shape), and the
+// small reduction kernels every backward uses.  bfloat16 inputs take the tensor-core kernels instead (the dZ
+// form of the encode kernel for pass A; the dQ and token kernels of the tensor-core backward for pass B when
+// D <= 32); the formulas are the same.
 //
 // The paper times a backward pass without writing it out; these kernels apply the chain rule to its encode and
 // decode equations (Section 3.2).  With S[m,n] = scale * q_m . k_n,
