@@ -4,9 +4,11 @@
 //   dS[m,n] = W_dec[n,m] (dY_n . Z_m - dd[n]) + W_enc[m,n] (dZ_m . V_n - de[m]),
 //   W_dec[n,m] = exp(S[m,n] - lse_dec[n]),  W_enc[m,n] = valid(n) exp(S[m,n] - lse_enc[m]),  S = scale * q_m . k_n.
 // The kernel has the shape of the encode kernel (latents on the 128 TMEM lanes, tokens on columns, the CTA's
-// token range split over N, one pipeline per softmax group with its own issuing warp): per unit of 32 tokens
+// token range split over N, one pipeline per softmax group with its own issuing warp): per unit of 16 tokens
 // three MMAs put S, A = Z dY^T and C = dZ V^T side by side in tensor memory, the group's threads turn them into
-// bf16 dS over the scores, and a fourth MMA adds dS K_unit to the group's partial dQ.  Z and dZ enter as two bf16
+// dS (two bf16 halves) over columns they have read, and two more MMAs add dS K_unit to the group's partial dQ.
+// Units alternate between two such buffers, so the tiles of the next unit and the dQ MMAs of the previous one
+// run while the group works on the current one (2 x 48 + D <= 128 columns per group).  Z and dZ enter as two bf16
 // halves each (hi + lo): the products dY.Z_m and dZ_m.V_n are differenced against dd and de.
 #pragma once
 
@@ -14,7 +16,7 @@
 
 namespace flare {
 
-constexpr int kBqStages = 2;     // (K, V, dY) tile triples in flight
+constexpr int kBqStages = 3;     // (K, V, dY) tile triples in flight
 
 struct BwdDqTcArgs {
     const float *Z, *dZ;       // [B,H,M,D]
@@ -36,7 +38,7 @@ struct BwdDqSmem {
     // Q, Z_hi, Z_lo, dZ_hi, dZ_lo: 256 latent rows each
     __host__ __device__ static size_t lat_off(int which) { return q_off() + (size_t)which * 2 * kTile * G::RB; }
     __host__ __device__ static size_t bar_off() { return lat_off(5); }
-    static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 3 * 32 * sizeof(float);   // per softmax warp: 3 x 32 column constants
+    static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 64 * sizeof(float);   // per softmax warp: 2 x 64 column constants
     __host__ __device__ static size_t col_off() { return bar_off() + 512; }
     __host__ __device__ static size_t total() {
         size_t t = col_off() + kColBytes + 1024;
@@ -57,8 +59,9 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint8_t *sQ = smem + SM::lat_off(0);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off());
     constexpr int NG = kSoftmaxGroups;
-    enum { T_FULL = 0, T_EMPTY = T_FULL + kBqStages, S_FULL = T_EMPTY + kBqStages, P_FULL = S_FULL + NG,
-           ACC_DONE = P_FULL + NG, Q_FULL = ACC_DONE + NG, NBARS };
+    // per group: S_FULL and P_FULL for each of its two unit buffers
+    enum { T_FULL = 0, T_EMPTY = T_FULL + kBqStages, S_FULL = T_EMPTY + kBqStages, P_FULL = S_FULL + 2 * NG,
+           ACC_DONE = P_FULL + 2 * NG, Q_FULL = ACC_DONE + NG, NBARS };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -74,15 +77,15 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
     const int rows_here = min(M - lb0 * kTile, 2 * kTile);
-    constexpr int SLOT_COLS = 256, HALF = kTile / 2, UNIT = 32;
+    constexpr int SLOT_COLS = 256, HALF = kTile / 2, UNIT = 16, UPH = HALF / UNIT;   // units per half tile
     constexpr uint32_t NCOLS = 512;
-    // per group (128 columns): S at 0, A at 32, C at 64, partial dQ at 96
+    // per group (128 columns): two unit buffers of 48 columns (S, A, C: 16 each), partial dQ at 96
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
 
     if (threadIdx.x == 0) {
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
-            ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + NG) ? 128u
+            ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? 128u
                                    : (i >= T_EMPTY && i < T_EMPTY + kBqStages) ? users : 1u);
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -144,48 +147,56 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 5; ++i) ldesc[i] = ptx::smem_desc(ptx::smem_u32(smem + SM::lat_off(i)), 16, G::SBO, G::SWZ) + blk;
             const uint32_t gcol = tm + j * SLOT_COLS + c * 2 * HALF;
-            const uint32_t dcol = gcol + 3 * UNIT;
+            const uint32_t dcol = gcol + 96;
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrBwdDq | 2);
             const int jobs = (nq - j + nslots - 1) / nslots;
-            const int units = 2 * jobs;
-            int t = alternate ? j : 0;
+            const int units = UPH * jobs;
+            // Order of issue, as in the encode kernel: the three tiles of units 0 and 1, then for every unit n its dQ
+            // MMAs as soon as its dS is handed over, then the tiles of unit n+2 into the buffer that dS has just left.
+            int t_s = alternate ? j : 0, t_v = t_s;                         // tiles of the next tile-unit / dQ-unit
             const int t_step = alternate ? 2 : 1;
-            for (int n = 0; ok && n < units; ++n) {
-                const int s = t % kBqStages, w = n & 1;
-                if (w == 0) {
-                    if (!ptx::mbar_wait(bar(T_FULL + s), (t / kBqStages) & 1, abort_flag, kErrBwdDq | 3)) break;
-                    ptx::tc_fence_after();
-                }
+            auto issue_tiles = [&](int n) -> bool {
+                const int s = t_s % kBqStages, w = n % UPH;
+                if (w == 0 && !ptx::mbar_wait(bar(T_FULL + s), (t_s / kBqStages) & 1, abort_flag, kErrBwdDq | 3)) return false;
+                ptx::tc_fence_after();
                 const uint32_t tbase = ptx::smem_u32(sT + (size_t)s * 3 * G::TILE_BYTES);
-                const uint64_t rowoff = (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);   // the unit's 32 token rows
+                const uint64_t rowoff = (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);   // the unit's 16 token rows
                 const uint64_t kdesc = ptx::smem_desc(tbase, 16, G::SBO, G::SWZ) + rowoff;
                 const uint64_t vdesc = ptx::smem_desc(tbase + G::TILE_BYTES, 16, G::SBO, G::SWZ) + rowoff;
                 const uint64_t gdesc = ptx::smem_desc(tbase + 2 * G::TILE_BYTES, 16, G::SBO, G::SWZ) + rowoff;
-                // S = Q K^T | A = (Z_hi + Z_lo) dY^T | C = (dZ_hi + dZ_lo) V^T, each 128 latents x 32 tokens
+                const uint32_t bcol = gcol + (n & 1) * 3 * UNIT;
+                // S = Q K^T | A = (Z_hi + Z_lo) dY^T | C = (dZ_hi + dZ_lo) V^T, each 128 latents x 16 tokens
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol, ldesc[0] + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(bcol, ldesc[0] + 2 * k, kdesc + 2 * k, idescS, k > 0);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + UNIT, ldesc[1] + 2 * k, gdesc + 2 * k, idescS, k > 0);
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(bcol + UNIT, ldesc[1] + 2 * k, gdesc + 2 * k, idescS, k > 0);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + UNIT, ldesc[2] + 2 * k, gdesc + 2 * k, idescS, 1u);
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(bcol + UNIT, ldesc[2] + 2 * k, gdesc + 2 * k, idescS, 1u);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + 2 * UNIT, ldesc[3] + 2 * k, vdesc + 2 * k, idescS, k > 0);
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(bcol + 2 * UNIT, ldesc[3] + 2 * k, vdesc + 2 * k, idescS, k > 0);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + 2 * UNIT, ldesc[4] + 2 * k, vdesc + 2 * k, idescS, 1u);
-                ptx::mma_commit(bar(S_FULL + g));
-                if (!ptx::mbar_wait(bar(P_FULL + g), n & 1, abort_flag, kErrBwdDq | 4)) break;
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(bcol + 2 * UNIT, ldesc[4] + 2 * k, vdesc + 2 * k, idescS, 1u);
+                ptx::mma_commit(bar(S_FULL + 2 * g + (n & 1)));
+                if (w == UPH - 1) t_s += t_step;
+                return true;
+            };
+            for (int n = 0; ok && n < 2 && n < units; ++n) ok = issue_tiles(n);
+            for (int n = 0; ok && n < units; ++n) {
+                const int s = t_v % kBqStages, w = n % UPH;
+                if (!ptx::mbar_wait(bar(P_FULL + 2 * g + (n & 1)), (n >> 1) & 1, abort_flag, kErrBwdDq | 4)) { ok = false; break; }
                 ptx::tc_fence_after();
-                // dQ_part += dS_unit K_unit: the K tile as the MN-major B operand, 16 token rows further on per k-step
-                const uint64_t kmn = ptx::smem_desc(tbase, G::SBO, G::SBO, G::SWZ) + rowoff;
-#pragma unroll
-                for (int k = 0; k < UNIT / 16; ++k)
-                    ptx::mma_ts(dcol, gcol + k * 8, kmn + (uint64_t)(k * G::RB), idescQ, (n > 0 || k > 0) ? 1u : 0u);
-#pragma unroll
-                for (int k = 0; k < UNIT / 16; ++k) ptx::mma_ts(dcol, gcol + UNIT + k * 8, kmn + (uint64_t)(k * G::RB), idescQ, 1u);
-                if (w == 1) {
+                // dQ_part += dS_unit K_unit (hi, then lo half of dS): the unit's 16 token rows of the K tile as the
+                // MN-major B operand
+                const uint64_t kmn = ptx::smem_desc(ptx::smem_u32(sT + (size_t)s * 3 * G::TILE_BYTES), G::SBO, G::SBO, G::SWZ) +
+                                     (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
+                const uint32_t bcol = gcol + (n & 1) * 3 * UNIT;
+                ptx::mma_ts(dcol, bcol, kmn, idescQ, n > 0 ? 1u : 0u);
+                ptx::mma_ts(dcol, bcol + UNIT, kmn, idescQ, 1u);
+                if (w == UPH - 1) {
                     ptx::mma_commit(bar(T_EMPTY + s));
-                    t += t_step;
+                    t_v += t_step;
                 }
+                if (n + 2 < units) ok = issue_tiles(n + 2);
             }
             if (ok) ptx::mma_commit(bar(ACC_DONE + g));
         }
@@ -195,7 +206,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int row = ((warp & 3) << 5) + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
         const uint32_t gcol = tm + lane_addr + j * SLOT_COLS + c * 2 * HALF;
-        const uint32_t abase = gcol + 3 * UNIT;
+        const uint32_t abase = gcol + 96;
         const float2 sl2p = make_float2(a.sl2, a.sl2);
         const int lb = alternate ? 0 : lb0 + j;
         const int m = lb * kTile + row;
@@ -208,41 +219,32 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             negde = -a.de[r];
         }
         const float2 neglep = make_float2(negle, negle), negdep = make_float2(negde, negde);
-        float *cst = reinterpret_cast<float *>(smem + SM::col_off()) + (warp - kFirstSoftmaxWarp) * 96;   // this warp's column constants
+        // this warp's column constants for the 64 tokens of its half tile: -lse_dec (log2 units), then -dd
+        float *cst = reinterpret_cast<float *>(smem + SM::col_off()) + (warp - kFirstSoftmaxWarp) * 128;
         int done = 0;
         bool ok = true;
-        auto unit = [&](auto masked, int t, int w) -> bool {
+        // One unit: 16 token columns on buffer (done & 1).  wv: validity bits of the 16 tokens (kMasked only).
+        auto unit = [&](auto masked, int w, uint32_t wv) -> bool {
             constexpr bool kMasked = decltype(masked)::value;
-            const int n = t * kTile + c * HALF + w * UNIT + lane;          // this lane fetches the constants of token n
-            uint32_t wv = 0xffffffffu;
-            __syncwarp();                                                   // the previous unit's reads are done
-            if (n < a.N) {
-                const size_t i = ((size_t)b * a.N + n) * a.H + h;
-                cst[lane] = -a.lse_dec[i] * 1.4426950408889634f;
-                cst[32 + lane] = -a.dd[i];
-            } else {
-                cst[lane] = -INFINITY;
-                cst[32 + lane] = 0.f;
-            }
-            if (kMasked) wv = __ballot_sync(0xffffffffu, n < a.N && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0));
-            __syncwarp();
-            if (!warp_wait(bar(S_FULL + g), done & 1, abort_flag, kErrBwdDq | 5)) return false;
+            const int buf = done & 1;
+            const uint32_t bcol = gcol + buf * 3 * UNIT;
+            if (!warp_wait(bar(S_FULL + 2 * g + buf), (done >> 1) & 1, abort_flag, kErrBwdDq | 5)) return false;
             ptx::tc_fence_after();
-            // 8 tokens at a time: their dS goes back as two bf16 halves, hi over score columns the thread has
-            // already read (4 packed columns per 8 tokens), lo likewise over the columns of A
+            // 8 tokens at a time: their dS goes back as two bf16 halves over columns the thread has already read
+            // (hi over S, lo over A: 4 packed columns per 8 tokens)
 #pragma unroll
-            for (int qd = 0; qd < 4; ++qd) {
+            for (int qd = 0; qd < 2; ++qd) {
                 uint32_t s[8], av[8], cv[8], pk[4], pl[4];
-                ptx::tmem_ld8(gcol + qd * 8, s);
-                ptx::tmem_ld8(gcol + UNIT + qd * 8, av);
-                ptx::tmem_ld8(gcol + 2 * UNIT + qd * 8, cv);
+                ptx::tmem_ld8(bcol + qd * 8, s);
+                ptx::tmem_ld8(bcol + UNIT + qd * 8, av);
+                ptx::tmem_ld8(bcol + 2 * UNIT + qd * 8, cv);
                 ptx::tmem_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const int col = qd * 8 + 2 * k;
                     const float2 sp = make_float2(__uint_as_float(s[2 * k]), __uint_as_float(s[2 * k + 1]));
-                    const float2 nld = *reinterpret_cast<const float2 *>(cst + col);
-                    const float2 ndd = *reinterpret_cast<const float2 *>(cst + 32 + col);
+                    const float2 nld = *reinterpret_cast<const float2 *>(cst + w * UNIT + col);
+                    const float2 ndd = *reinterpret_cast<const float2 *>(cst + HALF + w * UNIT + col);
                     const float2 xd = __ffma2_rn(sp, sl2p, nld), xe = __ffma2_rn(sp, sl2p, neglep);
                     const float2 pd = make_float2(ptx::ex2(xd.x), ptx::ex2(xd.y));
                     float2 pe = make_float2(ptx::ex2(xe.x), ptx::ex2(xe.y));
@@ -257,21 +259,52 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     pk[k] = hi;
                     pl[k] = ptx::pack_bf16(ds.x - __uint_as_float(hi << 16), ds.y - __uint_as_float(hi & 0xffff0000u));
                 }
-                ptx::tmem_st4(gcol + qd * 4, pk);
-                ptx::tmem_st4(gcol + UNIT + qd * 4, pl);
+                ptx::tmem_st4(bcol + qd * 4, pk);
+                ptx::tmem_st4(bcol + UNIT + qd * 4, pl);
             }
             ptx::tmem_wait_st();
             ptx::tc_fence_before();
-            ptx::mbar_arrive(bar(P_FULL + g));
+            ptx::mbar_arrive(bar(P_FULL + 2 * g + buf));
             ++done;
             return true;
         };
         if (j < nslots) {
+            // the constants of a tile are fetched one tile ahead (two tokens per lane) and parked, as loaded, in
+            // registers: nothing waits for the loads until the next tile begins
+            float f_ld[2], f_dd[2];
+            uint32_t f_ok[2];
+            auto fetch = [&](int t) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int n = t * kTile + c * HALF + e * 32 + lane;
+                    const bool in = n < a.N;
+                    const size_t i = ((size_t)b * a.N + (in ? n : 0)) * a.H + h;
+                    f_ld[e] = a.lse_dec[i];
+                    f_dd[e] = a.dd[i];
+                    f_ok[e] = a.key_mask == nullptr ? 1u : (uint32_t)a.key_mask[(size_t)b * a.N + (in ? n : 0)];
+                }
+            };
+            if (j < nq) fetch(t_begin + (alternate ? j : j / nslots));
             for (int q = j; ok && q < nq; q += nslots) {
                 const int t = t_begin + (alternate ? q : q / nslots);
                 const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;
+                __syncwarp();                                               // the previous tile's reads are done
+                bool v01[2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool in = t * kTile + c * HALF + e * 32 + lane < a.N;
+                    cst[e * 32 + lane] = in ? -f_ld[e] * 1.4426950408889634f : -INFINITY;
+                    cst[HALF + e * 32 + lane] = in ? -f_dd[e] : 0.f;
+                    v01[e] = in && f_ok[e] != 0;
+                }
+                const uint32_t wv0 = __ballot_sync(0xffffffffu, v01[0]), wv1 = __ballot_sync(0xffffffffu, v01[1]);
+                __syncwarp();
+                if (q + nslots < nq) fetch(t_begin + (alternate ? q + nslots : (q + nslots) / nslots));
 #pragma unroll 1
-                for (int w = 0; ok && w < 2; ++w) ok = plain ? unit(std::false_type{}, t, w) : unit(std::true_type{}, t, w);
+                for (int w = 0; ok && w < UPH; ++w) {
+                    const uint32_t wv = ((w < 2 ? wv0 : wv1) >> ((w & 1) * UNIT)) & 0xffffu;
+                    ok = plain ? unit(std::false_type{}, w, wv) : unit(std::true_type{}, w, wv);
+                }
             }
         }
         if (ok && j < nslots) ok = warp_wait(bar(ACC_DONE + g), 0, abort_flag, kErrBwdDq | 6);

@@ -224,13 +224,17 @@ def forward(Q, K, V, key_mask=None, scale=1.0, want_stats=False, stream=None):
     return (Y, Z, le, ld) if want_stats else Y
 
 
-def forward_backward(Q, K, V, dY, key_mask=None, scale=1.0, stream=None):
+def forward_backward(Q, K, V, dY, key_mask=None, scale=1.0, stream=None, check=False):
     """Convenience: flare_forward (keeping Z and the log-sum-exp rows) then flare_backward.
-    Returns (Y, dQ_lat [H,M,D] float32, dK, dV)."""
+    Returns (Y, dQ_lat [H,M,D] float32, dK, dV).  With check=True the stream is synchronised and a device-side
+    wait that gave up raises."""
     desc = make_desc(Q, K, scale)
     Y, Z, le, ld = forward(Q, K, V, key_mask, scale, want_stats=True, stream=stream)
     ws = alloc_workspace(desc, OP_BACKWARD, K.device)
     dQ = torch.empty(desc.H, desc.M, desc.D, dtype=torch.float32, device=K.device)
     dK, dV = torch.empty_like(K), torch.empty_like(V)
     flare_backward(desc, Q, K, V, key_mask, Y, dY, Z, le, ld, dQ, dK, dV, ws, stream)
+    if check:
+        (stream or torch.cuda.current_stream()).synchronize()
+        flare_check(ws, stream)
     return Y, dQ, dK, dV

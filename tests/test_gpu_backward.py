@@ -26,7 +26,7 @@ GRAD_TOL = {"f32": 1e-4, "bf16": 2e-2}
 
 def gpu_backward(inp, scale=1.0):
     Q, K, V, mask, dY = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask), dev(inp.dY)
-    Y, dQ, dK, dV = flare.forward_backward(Q, K, V, dY, mask, scale)
+    Y, dQ, dK, dV = flare.forward_backward(Q, K, V, dY, mask, scale, check=True)
     torch.cuda.synchronize()
     return dict(dQ=to_np64(dQ), dK=to_np64(dK), dV=to_np64(dV))
 
@@ -76,6 +76,9 @@ EDGE = [
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 600, 300, 64, "f32", 0.0),
     (1, 4, 64, 1, 16, "f32", 0.0),
+    # more (batch, head) pairs than SMs: every CTA walks several token tiles (one latent block / two)
+    (40, 4, 700, 64, 16, "bf16", 0.2),
+    (20, 8, 900, 256, 32, "bf16", 0.0),
 ]
 
 

@@ -55,7 +55,7 @@ def test_backward_full_size_padded(oracle):
     w = workloads.CONFIGS["padded"]
     inp = workloads.make_inputs(w)
     Q, K, V, mask, dY = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask), dev(inp.dY)
-    _, dQ, dK, dV = flare.forward_backward(Q, K, V, dY, mask, w.scale)
+    _, dQ, dK, dV = flare.forward_backward(Q, K, V, dY, mask, w.scale, check=True)
     torch.cuda.synchronize()
     ref = oracle.backward(to_np64(inp.Q), to_np64(inp.K), to_np64(inp.V), to_np64(inp.dY), key_mask=inp.key_mask.numpy(),
                           scale=w.scale)
