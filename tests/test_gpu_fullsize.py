@@ -50,13 +50,18 @@ def test_forward_full_size_sampled(oracle, w):
     assert_stored_close(Y_got, Y_ref, w.dtype, f"{w.name} Y (sampled rows)")
 
 
-def test_backward_full_size_padded(oracle):
-    """The long-sequence classification workload at full size: all three gradients, element by element."""
-    w = workloads.CONFIGS["padded"]
+BACKWARD_FULL = [workloads.CONFIGS["padded"], workloads.CONFIGS["mesh2d"].with_(backward=True),
+                 workloads.sweep_point(131072, 128)]
+
+
+@pytest.mark.parametrize("w", BACKWARD_FULL, ids=lambda w: w.name)
+def test_backward_full_size(oracle, w):
+    """Whole workloads at full size (the long-sequence classification batch, the 2-D mesh batch with its paired
+    heads, one long sequence): all three gradients, element by element."""
     inp = workloads.make_inputs(w)
     Q, K, V, mask, dY = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask), dev(inp.dY)
     _, dQ, dK, dV = flare.forward_backward(Q, K, V, dY, mask, w.scale, check=True)
     torch.cuda.synchronize()
-    ref = oracle.backward(to_np64(inp.Q), to_np64(inp.K), to_np64(inp.V), to_np64(inp.dY), key_mask=inp.key_mask.numpy(),
-                          scale=w.scale)
+    ref = oracle.backward(to_np64(inp.Q), to_np64(inp.K), to_np64(inp.V), to_np64(inp.dY),
+                          key_mask=None if inp.key_mask is None else inp.key_mask.numpy(), scale=w.scale)
     assert_grads_close(dict(dQ=to_np64(dQ), dK=to_np64(dK), dV=to_np64(dV)), ref, w.dtype, w.name)
