@@ -79,6 +79,11 @@ EDGE = [
     # more (batch, head) pairs than SMs: every CTA walks several token tiles (one latent block / two)
     (40, 4, 700, 64, 16, "bf16", 0.2),
     (20, 8, 900, 256, 32, "bf16", 0.0),
+    # latent counts that do not fill a unit of the tensor-core kernels, or leave a second latent block nearly empty
+    (2, 2, 300, 48, 16, "bf16", 0.1),
+    (1, 2, 200, 16, 32, "bf16", 0.0),
+    (1, 1, 130, 144, 32, "bf16", 0.0),
+    (1, 2, 260, 400, 16, "bf16", 0.3),
 ]
 
 
