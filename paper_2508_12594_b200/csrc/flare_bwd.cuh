@@ -144,7 +144,7 @@ bwd_token_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T 
             dd = fmaf(wdec, a, dd);
         }
     }
-    if (live) dd_out[((size_t)b * N + n) * H + h] = dd;
+    if (live) dd_out[((size_t)b * H + h) * N + n] = dd;
     for (int m0 = 0; m0 < M; m0 += kBwdLatents) {
         const int mc = min(kBwdLatents, M - m0);
         __syncthreads();
@@ -241,7 +241,7 @@ bwd_dq_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
             if (threadIdx.x < kBwdTileN) {
                 const int j = threadIdx.x, n = t0 + j;
                 const bool in = n < n1;
-                sDd[j] = in ? dd[((size_t)b * N + n) * H + h] : 0.f;
+                sDd[j] = in ? dd[((size_t)b * H + h) * N + n] : 0.f;
                 sLd[j] = in ? lse_dec[((size_t)b * N + n) * H + h] : INFINITY;
                 sValid[j] = in && (key_mask == nullptr || key_mask[(size_t)b * N + n] != 0);
             }

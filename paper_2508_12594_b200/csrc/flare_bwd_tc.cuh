@@ -21,7 +21,8 @@ constexpr int kBqStages = 3;     // (K, V, dY) tile triples in flight
 struct BwdDqTcArgs {
     const float *Z, *dZ;       // [B,H,M,D]
     const float *lse_enc, *de; // [B,H,M]
-    const float *lse_dec, *dd; // [B,N,H]
+    const float *lse_dec;      // [B,N,H]
+    const float *dd;           // [B,H,N] (workspace)
     const uint8_t *key_mask;   // [B,N] or null
     float *part;               // [P][B*H*M][D] partial dQ rows (un-scaled)
     uint32_t *status;
@@ -280,7 +281,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     const bool in = n < a.N;
                     const size_t i = ((size_t)b * a.N + (in ? n : 0)) * a.H + h;
                     f_ld[e] = a.lse_dec[i];
-                    f_dd[e] = a.dd[i];
+                    f_dd[e] = a.dd[((size_t)b * a.H + h) * a.N + (in ? n : 0)];
                     f_ok[e] = a.key_mask == nullptr ? 1u : (uint32_t)a.key_mask[(size_t)b * a.N + (in ? n : 0)];
                 }
             };
@@ -356,7 +357,7 @@ struct BwdTokTcArgs {
     const float *lse_dec;      // [B,N,H]
     const uint8_t *key_mask;   // [B,N] or null
     __nv_bfloat16 *dK, *dV;    // [B,N,H,D]
-    float *dd;                 // [B,N,H] out
+    float *dd;                 // [B,H,N] out (workspace)
     uint32_t *status;
     int B, H, N, M;
     float scale, sl2;
@@ -555,13 +556,60 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         uint32_t cnt = 0;
         int k_tile = 0;
         bool ok = true;
+        // The rows of a tile are written one sweep late: while the issuing warp finishes the tile's last MMAs the
+        // group already works on the first sweep of its next tile, whose MMAs do not touch the accumulators.
+        bool pend = false, p_inside = false;
+        size_t p_tok = 0, p_ddi = 0;
+        float p_dd = 0.f;
+        int p_k = 0;
+        auto write_rows = [&]() -> bool {
+            if (!warp_wait(bar(ACC_FULL + g), p_k & 1, abort_flag, kErrBwdTok | 8)) return false;
+            ptx::tc_fence_after();
+            uint32_t ak[D], avv[D];
+#pragma unroll
+            for (int dc = 0; dc < D / 16; ++dc) {
+                ptx::tmem_ld16(kcol + dc * 16, ak + dc * 16);
+                ptx::tmem_ld16(vcol + dc * 16, avv + dc * 16);
+            }
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(bar(ACC_FREE + g));
+            if (p_inside) {
+                a.dd[p_ddi] = p_dd;
+                uint4 *dk = reinterpret_cast<uint4 *>(a.dK + p_tok * D), *dv = reinterpret_cast<uint4 *>(a.dV + p_tok * D);
+#pragma unroll
+                for (int q = 0; q < D / 8; ++q) {
+                    uint32_t wk[4], wv4[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        wk[k] = ptx::pack_bf16(__uint_as_float(ak[8 * q + 2 * k]) * a.scale, __uint_as_float(ak[8 * q + 2 * k + 1]) * a.scale);
+                        wv4[k] = ptx::pack_bf16(__uint_as_float(avv[8 * q + 2 * k]), __uint_as_float(avv[8 * q + 2 * k + 1]));
+                    }
+                    dk[q] = make_uint4(wk[0], wk[1], wk[2], wk[3]);
+                    dv[q] = make_uint4(wv4[0], wv4[1], wv4[2], wv4[3]);
+                }
+            }
+            pend = false;
+            return true;
+        };
+        // this lane's token of a tile: its decode log-sum-exp and mask byte, fetched one tile ahead
+        float f_ld = 0.f;
+        uint32_t f_mask = 1u;
+        auto fetch = [&](int i) {
+            const int n = (blockIdx.x + i * gridDim.x) * kTile + row;
+            const size_t nn = (size_t)b * a.N + (n < a.N ? n : 0);
+            f_ld = a.lse_dec[nn * a.H + h];
+            f_mask = a.key_mask == nullptr ? 1u : (uint32_t)a.key_mask[nn];
+        };
+        if (g < ng && g < nt) fetch(g);
         for (int i = g; ok && g < ng && i < nt; i += ng, ++k_tile) {
             const int t = blockIdx.x + i * gridDim.x, n = t * kTile + row;
             const bool inside = n < a.N;
-            const bool valid = inside && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0);
+            const bool valid = inside && f_mask != 0;
             const size_t tok = ((size_t)b * a.N + (inside ? n : 0)) * a.H + h;
-            const float negld = inside ? -a.lse_dec[tok] * 1.4426950408889634f : -INFINITY;
+            const float negld = inside ? -f_ld * 1.4426950408889634f : -INFINITY;
             const float2 negldp = make_float2(negld, negld);
+            if (i + ng < nt) fetch(i + ng);
             const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;      // uniform over the group
             // sweep 1: dd[n] = sum_m W_dec[n,m] (dY_n . Z_m)
             float2 dd2 = make_float2(0.f, 0.f);
@@ -587,6 +635,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             }
             const float dd = dd2.x + dd2.y;
             const float2 negddp = make_float2(-dd, -dd);
+            if (ok && pend) ok = write_rows();                  // the previous tile's rows
             // sweep 2: dS^T and W_enc^T of every unit, handed to the issuing warp
             auto unit2 = [&](auto masked, int u) {
                 constexpr bool kMasked = decltype(masked)::value;
@@ -636,33 +685,10 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 ptx::mbar_arrive(bar(P_FULL + g));
             }
             if (!ok) break;
-            if (!warp_wait(bar(ACC_FULL + g), k_tile & 1, abort_flag, kErrBwdTok | 8)) { ok = false; break; }
-            ptx::tc_fence_after();
-            uint32_t ak[D], avv[D];
-#pragma unroll
-            for (int dc = 0; dc < D / 16; ++dc) {
-                ptx::tmem_ld16(kcol + dc * 16, ak + dc * 16);
-                ptx::tmem_ld16(vcol + dc * 16, avv + dc * 16);
-            }
-            ptx::tmem_wait_ld();
-            ptx::tc_fence_before();
-            ptx::mbar_arrive(bar(ACC_FREE + g));
-            if (inside) {
-                a.dd[tok] = dd;
-                uint4 *dk = reinterpret_cast<uint4 *>(a.dK + tok * D), *dv = reinterpret_cast<uint4 *>(a.dV + tok * D);
-#pragma unroll
-                for (int q = 0; q < D / 8; ++q) {
-                    uint32_t wk[4], wv4[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        wk[k] = ptx::pack_bf16(__uint_as_float(ak[8 * q + 2 * k]) * a.scale, __uint_as_float(ak[8 * q + 2 * k + 1]) * a.scale);
-                        wv4[k] = ptx::pack_bf16(__uint_as_float(avv[8 * q + 2 * k]), __uint_as_float(avv[8 * q + 2 * k + 1]));
-                    }
-                    dk[q] = make_uint4(wk[0], wk[1], wk[2], wk[3]);
-                    dv[q] = make_uint4(wv4[0], wv4[1], wv4[2], wv4[3]);
-                }
-            }
+            pend = true; p_inside = inside; p_tok = tok; p_dd = dd; p_k = k_tile;
+            p_ddi = ((size_t)b * a.H + h) * a.N + (inside ? n : 0);
         }
+        if (ok && pend) ok = write_rows();
     }
     ptx::tc_fence_before();
     __syncthreads();
