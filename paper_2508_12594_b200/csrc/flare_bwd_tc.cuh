@@ -19,6 +19,7 @@ namespace flare {
 constexpr int kBqStages = 3;     // (K, V, dY) tile triples in flight
 
 struct BwdDqTcArgs {
+    const __nv_bfloat16 *Q;    // [H,M,D] (read directly in the half-width form)
     const float *Z, *dZ;       // [B,H,M,D]
     const float *lse_enc, *de; // [B,H,M]
     const float *lse_dec;      // [B,N,H]
@@ -47,13 +48,16 @@ struct BwdDqSmem {
     }
 };
 
-// grid = (splits, H * pairs, B), as the encode kernel.
-template <int D>
+// grid = (splits, H * pairs, B), as the encode kernel.  kHalf: the half-width form of the forward kernels (the head
+// is DR = D/2 wide in memory; token tiles carry the next head's features in their upper half, every latent
+// operand zeros, and the upper half of the partial dQ is dropped).
+template <int D, bool kHalf = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdDqTcArgs a) {
     using G = TileGeom<D>;
     using SM = BwdDqSmem<D>;
+    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sT = smem + SM::tile_off;
@@ -96,14 +100,23 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         ptx::prefetch_tensormap(&tmQ);
     }
     if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), NCOLS);
-    // zero the latent rows beyond M (all five operands), then Z and dZ as bf16 hi/lo rows in the swizzled layout
+    // zero the latent rows beyond M (all five operands; in the half-width form all rows, whose upper halves stay
+    // zero), then Z and dZ as bf16 hi/lo rows in the swizzled layout
     for (int i = threadIdx.x; i < 5 * 2 * kTile * (G::RB / 16); i += kTcThreads) {
         const int which = i / (2 * kTile * (G::RB / 16)), rem = i % (2 * kTile * (G::RB / 16));
-        if (rem / (G::RB / 16) >= rows_here) reinterpret_cast<uint4 *>(smem + SM::lat_off(which))[rem] = make_uint4(0, 0, 0, 0);
+        if (kHalf || rem / (G::RB / 16) >= rows_here) reinterpret_cast<uint4 *>(smem + SM::lat_off(which))[rem] = make_uint4(0, 0, 0, 0);
     }
-    for (int i = threadIdx.x; i < 2 * rows_here * (D / 8); i += kTcThreads) {
-        const int which = i / (rows_here * (D / 8)), rem = i % (rows_here * (D / 8)), m = rem / (D / 8), ch = rem % (D / 8);
-        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + lb0 * kTile + m) * D + ch * 8;
+    if (kHalf) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < rows_here * (DR / 8); i += kTcThreads) {
+            const int m = i / (DR / 8), ch = i % (DR / 8);
+            *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
+                *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
+        }
+    }
+    for (int i = threadIdx.x; i < 2 * rows_here * (DR / 8); i += kTcThreads) {
+        const int which = i / (rows_here * (DR / 8)), rem = i % (rows_here * (DR / 8)), m = rem / (DR / 8), ch = rem % (DR / 8);
+        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + lb0 * kTile + m) * DR + ch * 8;
         const float4 lo4 = *reinterpret_cast<const float4 *>(src), hi4 = *reinterpret_cast<const float4 *>(src + 4);
         const float z[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
         uint32_t vh[4], vl[4];
@@ -124,17 +137,21 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(rows_here * G::RB));
-            for (int r = 0; r < rows_here; r += 16)
-                ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
+            if (kHalf) {
+                ptx::mbar_arrive(bar(Q_FULL));                  // Q was written by the threads before the block barrier
+            } else {
+                ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(rows_here * G::RB));
+                for (int r = 0; r < rows_here; r += 16)
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
+            }
             for (int i = 0; i < nt; ++i) {
                 const int s = i % kBqStages;
                 if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / kBqStages) & 1) ^ 1, abort_flag, kErrBwdDq | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(T_FULL + s), 3 * G::TILE_BYTES);
                 uint8_t *dst = sT + (size_t)s * 3 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * D, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * D, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * D, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * DR, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * DR, (t_begin + i) * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -322,9 +339,9 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (ok && j < nslots && m < M) {
             const long rows = (long)a.B * a.H * M;
             const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);
-            float4 *dst = reinterpret_cast<float4 *>(a.part + ((size_t)part * rows + ((size_t)b * a.H + h) * M + m) * D);
+            float4 *dst = reinterpret_cast<float4 *>(a.part + ((size_t)part * rows + ((size_t)b * a.H + h) * M + m) * DR);
 #pragma unroll
-            for (int dc = 0; dc < D / 4; ++dc)
+            for (int dc = 0; dc < DR / 4; ++dc)
                 dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
                                       __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
         }
@@ -352,6 +369,7 @@ struct BwdTokGeom {
 };
 
 struct BwdTokTcArgs {
+    const __nv_bfloat16 *Q;    // [H,M,D] (read directly in the half-width form)
     const float *Z, *dZ;       // [B,H,M,D]
     const float *lse_enc, *de; // [B,H,M]
     const float *lse_dec;      // [B,N,H]
@@ -387,7 +405,8 @@ struct BwdTokSmem {
 };
 
 // grid = (CTAs per head, H, B); a CTA takes the token tiles blockIdx.x, blockIdx.x + gridDim.x, ...
-template <int D>
+// kHalf: the half-width form (head DR = D/2 wide in memory; the upper halves of the rows of dK and dV are dropped).
+template <int D, bool kHalf = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdTokTcArgs a) {
@@ -395,6 +414,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     using SM = BwdTokSmem<D>;
     constexpr int UNIT = BwdTokGeom<D>::kUnit;
     constexpr int kMaxSt = BwdTokGeom<D>::kMaxStages;
+    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int M = a.M, MU = SM::padded_m(M), stages = a.stages;
@@ -427,9 +447,18 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), NCOLS);
     // latent rows M..MU-1 of all five operands are zero; their columns carry -lse_enc = -inf
-    for (int i = threadIdx.x; i < 5 * (MU - M) * (G::RB / 16); i += kTcThreads) {
-        const int which = i / ((MU - M) * (G::RB / 16)), rem = i % ((MU - M) * (G::RB / 16));
-        reinterpret_cast<uint4 *>(smem + SM::lat_off(stages, M, which) + (size_t)M * G::RB)[rem] = make_uint4(0, 0, 0, 0);
+    const int zfirst = kHalf ? 0 : M;                           // half-width form: every row, whose upper half stays zero
+    for (int i = threadIdx.x; i < 5 * (MU - zfirst) * (G::RB / 16); i += kTcThreads) {
+        const int which = i / ((MU - zfirst) * (G::RB / 16)), rem = i % ((MU - zfirst) * (G::RB / 16));
+        reinterpret_cast<uint4 *>(smem + SM::lat_off(stages, M, which) + (size_t)zfirst * G::RB)[rem] = make_uint4(0, 0, 0, 0);
+    }
+    if (kHalf) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+            const int m = i / (DR / 8), ch = i % (DR / 8);
+            *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
+                *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + ch * 8);
+        }
     }
     for (int m = threadIdx.x; m < MU; m += kTcThreads) {
         float nle = -INFINITY, nde = 0.f;
@@ -442,9 +471,9 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         cst[m] = nle;
         cst[MU + m] = nde;
     }
-    for (int i = threadIdx.x; i < 2 * M * (D / 8); i += kTcThreads) {
-        const int which = i / (M * (D / 8)), rem = i % (M * (D / 8)), m = rem / (D / 8), ch = rem % (D / 8);
-        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + m) * D + ch * 8;
+    for (int i = threadIdx.x; i < 2 * M * (DR / 8); i += kTcThreads) {
+        const int which = i / (M * (DR / 8)), rem = i % (M * (DR / 8)), m = rem / (DR / 8), ch = rem % (DR / 8);
+        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + m) * DR + ch * 8;
         const float4 lo4 = *reinterpret_cast<const float4 *>(src), hi4 = *reinterpret_cast<const float4 *>(src + 4);
         const float z[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
         uint32_t vh[4], vl[4];
@@ -465,17 +494,21 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
     if (warp == 0) {
         if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
-            for (int r = 0; r < M; r += 16)
-                ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+            if (kHalf) {
+                ptx::mbar_arrive(bar(Q_FULL));                  // Q was written by the threads before the block barrier
+            } else {
+                ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
+                for (int r = 0; r < M; r += 16)
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+            }
             for (int i = 0; i < nt; ++i) {
                 const int s = i % stages, t = blockIdx.x + i * gridDim.x;
                 if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / stages) & 1) ^ 1, abort_flag, kErrBwdTok | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(T_FULL + s), 3 * G::TILE_BYTES);
                 uint8_t *dst = smem + (size_t)s * 3 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * D, t * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * D, t * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * D, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * DR, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * DR, t * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -576,9 +609,9 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             ptx::mbar_arrive(bar(ACC_FREE + g));
             if (p_inside) {
                 a.dd[p_ddi] = p_dd;
-                uint4 *dk = reinterpret_cast<uint4 *>(a.dK + p_tok * D), *dv = reinterpret_cast<uint4 *>(a.dV + p_tok * D);
+                uint4 *dk = reinterpret_cast<uint4 *>(a.dK + p_tok * DR), *dv = reinterpret_cast<uint4 *>(a.dV + p_tok * DR);
 #pragma unroll
-                for (int q = 0; q < D / 8; ++q) {
+                for (int q = 0; q < DR / 8; ++q) {
                     uint32_t wk[4], wv4[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {

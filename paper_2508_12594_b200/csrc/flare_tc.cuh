@@ -176,6 +176,7 @@ inline DecodePlan make_decode_plan(int M, int D) {
 }
 
 struct DecodeTcArgs {
+    const __nv_bfloat16 *Q;  // [H,M,D] (read directly in the half-width form)
     const float *Z;      // [B,H,M,D]
     __nv_bfloat16 *Y;    // [B,N,H,D]
     float *lse_dec;      // [B,N,H] or null
@@ -212,9 +213,15 @@ struct DecodeSmem {
 
 // Decode.  grid = (ctas_per_head, H, B); each CTA walks a contiguous range of 128-token tiles of one (b, h)
 // with Q_h and Z_bh resident in shared memory.
-template <int D>
+//
+// Half-width form (kHalf): the head is DR = D/2 wide in memory.  The kernel still multiplies D-wide rows: a token
+// row of the K tile is the head's DR features followed by the next head's (or zeros past the last head), the rows
+// of Q and Z are staged with zeros in their upper half, so the neighbour's features meet zeros in every product.
+// This is how a head width of 8 (the smallest MMA K-step is 16) runs on the tensor cores.
+template <int D, bool kHalf = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
+    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
     using G = TileGeom<D>;
     using SM = DecodeSmem<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -268,11 +275,24 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // Z_bh -> two bf16 halves (hi = round(z), lo = round(z - hi)); rows of RB bytes in the swizzled layout the
     // MMA's B operand expects (latent-major rows), the lo half M rows after the hi half.
     {
-        const float *Zg = a.Z + ((size_t)b * a.H + h) * M * D;
-        for (int i = threadIdx.x; i < M * (D / 8); i += kTcThreads) {
-            const int m = i / (D / 8), c = i % (D / 8);
-            const float4 lo = *reinterpret_cast<const float4 *>(Zg + (size_t)m * D + c * 8);
-            const float4 hi = *reinterpret_cast<const float4 *>(Zg + (size_t)m * D + c * 8 + 4);
+        const float *Zg = a.Z + ((size_t)b * a.H + h) * M * DR;
+        if (kHalf) {   // upper halves of the rows of Q, Z_hi and Z_lo are zero
+            for (int i = threadIdx.x; i < M * (D / 8); i += kTcThreads) {
+                reinterpret_cast<uint4 *>(sQ)[i] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4 *>(sZ)[i] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4 *>(sZ + (size_t)M * G::RB)[i] = make_uint4(0, 0, 0, 0);
+            }
+            __syncthreads();
+            for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+                const int m = i / (DR / 8), c = i % (DR / 8);
+                *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) =
+                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + c * 8);
+            }
+        }
+        for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+            const int m = i / (DR / 8), c = i % (DR / 8);
+            const float4 lo = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8);
+            const float4 hi = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8 + 4);
             const float z[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
             uint32_t vh[4], vl[4];
 #pragma unroll
@@ -295,15 +315,19 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {
-            // Q_h: M/16 boxes of 16 rows
-            ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
-            for (int r = 0; r < M; r += 16)
-                ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+            if (kHalf) {
+                ptx::mbar_arrive(bar(Q_FULL));                  // Q was written by the threads before the block barrier
+            } else {
+                // Q_h: M/16 boxes of 16 rows
+                ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
+                for (int r = 0; r < M; r += 16)
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+            }
             for (int i = 0; i < ntiles; ++i) {
                 const int s = i % nstages;
                 if (!ptx::mbar_wait(bar(K_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrDecode | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(K_FULL + s), G::TILE_BYTES);
-                ptx::tma_load_3d(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), &tmK, bar(K_FULL + s), h * D,
+                ptx::tma_load_3d(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), &tmK, bar(K_FULL + s), h * DR,
                                  (t_begin + i) * kTile, b);
             }
         }
@@ -452,7 +476,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             const float inv = 1.f / ltot;
             const int n = (t_begin + i) * kTile + row;
-            uint4 *dst = reinterpret_cast<uint4 *>(a.Y + (((size_t)b * a.N + (n < a.N ? n : 0)) * a.H + h) * D);
+            uint4 *dst = reinterpret_cast<uint4 *>(a.Y + (((size_t)b * a.N + (n < a.N ? n : 0)) * a.H + h) * DR);
 #pragma unroll
             for (int dc = 0; dc < D / 16; ++dc) {
                 float y[16];
@@ -474,9 +498,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (n < a.N) {
                     dst[2 * dc] = make_uint4(ptx::pack_bf16(y[0] * inv, y[1] * inv), ptx::pack_bf16(y[2] * inv, y[3] * inv),
                                              ptx::pack_bf16(y[4] * inv, y[5] * inv), ptx::pack_bf16(y[6] * inv, y[7] * inv));
-                    dst[2 * dc + 1] =
-                        make_uint4(ptx::pack_bf16(y[8] * inv, y[9] * inv), ptx::pack_bf16(y[10] * inv, y[11] * inv),
-                                   ptx::pack_bf16(y[12] * inv, y[13] * inv), ptx::pack_bf16(y[14] * inv, y[15] * inv));
+                    if (DR > 8 + 16 * dc)
+                        dst[2 * dc + 1] =
+                            make_uint4(ptx::pack_bf16(y[8] * inv, y[9] * inv), ptx::pack_bf16(y[10] * inv, y[11] * inv),
+                                       ptx::pack_bf16(y[12] * inv, y[13] * inv), ptx::pack_bf16(y[14] * inv, y[15] * inv));
                 }
             }
             ptx::tc_fence_before();
@@ -545,11 +570,17 @@ struct EncodeSmem {
 // the encode weights, dZ_m = sum_n exp(S[m,n] - lse_dec[n]) dY_n.  Every column (token) carries its own shift
 // and the weights are already normalised, so there is no running maximum, no rescaling and no sum; tokens
 // beyond N get the shift -inf.  Every group leaves one partial sum of dZ per split (part_acc).
-template <int D, bool kPair, bool kDz = false>
+//
+// Half-width form (kHalf; not with kPair): the head is DR = D/2 wide in memory, as in the decode kernel: K and V
+// tile rows carry the next head's features in their upper half, Q rows zeros; the upper half of the accumulator
+// (weights times the neighbour's values) is dropped.
+template <int D, bool kPair, bool kDz = false, bool kHalf = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
+    static_assert(!(kPair && kHalf), "head pairing and the half-width form exclude each other");
     constexpr int DG = kPair ? 2 * D : D;
+    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
     using G = TileGeom<DG>;
     using SM = EncodeSmem<DG>;
     extern __shared__ uint8_t smem_raw[];
@@ -577,7 +608,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int lb0 = pair * 2;                                   // latent block of slot 0
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
-    const int rows_here = kPair ? 0 : min(M - lb0 * kTile, 2 * kTile);   // latent rows of Q_h fetched by TMA
+    const int rows_q = min(M - lb0 * kTile, 2 * kTile);                  // latent rows of this CTA
+    const int rows_here = (kPair || kHalf) ? 0 : rows_q;                 // ... fetched by TMA
     constexpr int SLOT_COLS = 256;   // per slot and half (128 columns): two score buffers of UNIT columns, accumulator at 64
     constexpr int HALF = kTile / 2;
     constexpr int UNIT = 32;         // tokens per unit of work of a group
@@ -611,6 +643,15 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             *reinterpret_cast<uint4 *>(sQ + (size_t)r * G::RB + ((chunk ^ G::swz(r)) << 4)) = v;
         }
     }
+    if (kHalf) {
+        // rows [Q[h][m] | 0]: the lower DR/8 chunks of every row, the rest stays zero
+        __syncthreads();
+        for (int i = threadIdx.x; i < rows_q * (DR / 8); i += kTcThreads) {
+            const int m = i / (DR / 8), ch = i % (DR / 8);
+            *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
+                *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
+        }
+    }
     ptx::fence_proxy_async_smem();
     ptx::tc_fence_before();
     __syncthreads();
@@ -619,7 +660,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {
-            if (kPair) {
+            if (kPair || kHalf) {
                 ptx::mbar_arrive(bar(Q_FULL));                  // Q was written by the threads before the block barrier
             } else {
                 ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(rows_here * G::RB));
@@ -631,8 +672,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (!ptx::mbar_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(KV_FULL + s), 2 * G::TILE_BYTES);
                 uint8_t *dst = sKV + (size_t)s * 2 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(KV_FULL + s), h * D, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * D, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(KV_FULL + s), h * DR, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR, (t_begin + i) * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -814,9 +855,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 a.part_m[prow] = (m_run == -INFINITY) ? -INFINITY : m_run * a.scale;
                 a.part_l[prow] = l2.x + l2.y;
             }
-            float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * D);
+            float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * DR);
 #pragma unroll
-            for (int dc = 0; dc < D / 4; ++dc)
+            for (int dc = 0; dc < DR / 4; ++dc)
                 dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
                                       __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
         }

@@ -84,6 +84,11 @@ EDGE = [
     (1, 2, 200, 16, 32, "bf16", 0.0),
     (1, 1, 130, 144, 32, "bf16", 0.0),
     (1, 2, 260, 400, 16, "bf16", 0.3),
+    # head width 8 on the tensor cores (token tiles span two heads), with an odd head count and a single head
+    (2, 4, 600, 48, 8, "bf16", 0.1),
+    (1, 3, 700, 256, 8, "bf16", 0.0),
+    (24, 8, 500, 64, 8, "bf16", 0.2),
+    (1, 1, 200, 32, 8, "bf16", 0.0),
 ]
 
 

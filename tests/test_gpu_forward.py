@@ -48,6 +48,12 @@ EDGE = [
     (2, 3, 1100, 32, 16, "bf16", 0.2),     # odd head count: one head per CTA although M <= 64
     (1, 4, 900, 16, 16, "bf16", 0.0),      # two heads per CTA, most latent lanes empty
     (1, 6, 450, 64, 32, "bf16", 0.3),      # two heads per CTA, all lanes in use, padding
+    # head width 8 on the tensor cores: token tiles of 16 columns span two heads (the last head's upper half lies
+    # beyond the tensor); a single head stays on the CUDA cores
+    (2, 4, 1100, 64, 8, "bf16", 0.2),
+    (1, 3, 900, 256, 8, "bf16", 0.0),
+    (1, 2, 700, 400, 8, "bf16", 0.0),
+    (1, 1, 300, 32, 8, "bf16", 0.0),
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 2049, 300, 64, "f32", 0.0),
     (1, 4, 64, 1, 16, "f32", 0.0),
