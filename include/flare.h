@@ -29,7 +29,7 @@
  * run concurrently on different streams only with different workspaces.  Results are bitwise reproducible
  * for a fixed descriptor on a fixed device.
  *
- * Supported shapes: D in {8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 512.
+ * Supported shapes: D in {4, 8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 512.
  * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation (D = 8 as the lower half of a
  * 16-wide product whose upper half meets zeros; with a single head of width 8, on the CUDA cores).
  *

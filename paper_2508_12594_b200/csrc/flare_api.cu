@@ -67,7 +67,7 @@ int check_desc(const flare_desc_t *d) {
     if (d->B <= 0 || d->H <= 0 || d->N <= 0 || d->M <= 0 || d->D <= 0) return FLARE_ERR_INVALID_ARG;
     if (!std::isfinite(d->scale)) return FLARE_ERR_INVALID_ARG;
     if (d->dtype != FLARE_DTYPE_F32 && d->dtype != FLARE_DTYPE_BF16) return FLARE_ERR_UNSUPPORTED;
-    if (d->D != 8 && d->D != 16 && d->D != 32 && d->D != 64) return FLARE_ERR_UNSUPPORTED;
+    if (d->D != 4 && d->D != 8 && d->D != 16 && d->D != 32 && d->D != 64) return FLARE_ERR_UNSUPPORTED;
     if (d->dtype == FLARE_DTYPE_BF16 && (d->M % 16 != 0 || d->M < 16 || d->M > 512)) return FLARE_ERR_UNSUPPORTED;
     if ((long)d->B * d->N > (1L << 31) - 1 || d->H > 65535 || d->B > 65535) return FLARE_ERR_UNSUPPORTED;
     return FLARE_OK;
@@ -338,7 +338,7 @@ int launch_encode_simt(const flare_desc_t *d, const SimtPlan &p, const void *Q, 
                                                           pacc, d->B, d->H, d->N, d->M, p.LM, p.chunk, d->scale); \
         break;
     switch (d->D) {
-        FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
+        FLARE_CASE(4) FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
         default: return FLARE_ERR_UNSUPPORTED;
     }
 #undef FLARE_CASE
@@ -356,7 +356,7 @@ int launch_decode_simt(const flare_desc_t *d, const void *Q, const void *K, cons
                                                           d->N, d->M, d->scale);                                  \
         break;
     switch (d->D) {
-        FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
+        FLARE_CASE(4) FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
         default: return FLARE_ERR_UNSUPPORTED;
     }
 #undef FLARE_CASE
@@ -432,7 +432,7 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     FLARE_CUDA(cudaMemsetAsync(ws, 0, kHeaderBytes, st));
     int dz_parts = pa.P;
     bool dz_on_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && D >= 8) {
         if (bwd_dz_on_tensor_cores(d)) {
             const TcEncodePlan tp = tc_encode_plan(d, sms);
             uint32_t *status = reinterpret_cast<uint32_t *>(ws);
@@ -461,7 +461,7 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     bwd_de_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(dZ, Z, de, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
     bool tok_on_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value && D <= 32) {
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && D >= 8 && D <= 32) {
         constexpr int DK = D == 8 ? 16 : D;                     // width the kernels multiply (D = 8: half-width form)
         if (bwd_dq_on_tensor_cores(d) && BwdTokSmem<DK>::stages(d->M) >= 1) {
             const int rc = launch_bwd_token_tc<DK, D == 8>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd,
@@ -478,7 +478,7 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     }
     int dq_parts = pb.P;
     bool dq_on_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value && D <= 32) {
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && D >= 8 && D <= 32) {
         if (bwd_dq_on_tensor_cores(d)) {
             const int rc = launch_bwd_dq_tc<D == 8 ? 16 : D, D == 8>(d, tc_dq_plan(d, sms), Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part,
                                                reinterpret_cast<uint32_t *>(ws), st);
@@ -512,6 +512,7 @@ int backward_simt(const flare_desc_t *d, int sms, const void *Q, const void *K, 
                   const void *Y, const void *dY, const float *Z, const float *lse_enc, const float *lse_dec, float *dQ,
                   void *dK, void *dV, char *ws, cudaStream_t st) {
     switch (d->D) {
+        case 4: return launch_backward_simt<T, 4>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
         case 8: return launch_backward_simt<T, 8>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
         case 16: return launch_backward_simt<T, 16>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
         case 32: return launch_backward_simt<T, 32>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);

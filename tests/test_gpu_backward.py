@@ -89,6 +89,10 @@ EDGE = [
     (1, 3, 700, 256, 8, "bf16", 0.0),
     (24, 8, 500, 64, 8, "bf16", 0.2),
     (1, 1, 200, 32, 8, "bf16", 0.0),
+    # head width 4
+    (2, 4, 300, 32, 4, "bf16", 0.1),
+    (1, 16, 500, 64, 4, "bf16", 0.0),
+    (1, 2, 200, 7, 4, "f32", 0.0),
 ]
 
 

@@ -54,6 +54,10 @@ EDGE = [
     (1, 3, 900, 256, 8, "bf16", 0.0),
     (1, 2, 700, 400, 8, "bf16", 0.0),
     (1, 1, 300, 32, 8, "bf16", 0.0),
+    # head width 4 (the paper's other setting for its PDE models)
+    (2, 4, 300, 32, 4, "bf16", 0.1),
+    (1, 16, 700, 64, 4, "bf16", 0.0),
+    (1, 2, 200, 7, 4, "f32", 0.0),
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 2049, 300, 64, "f32", 0.0),
     (1, 4, 64, 1, 16, "f32", 0.0),
