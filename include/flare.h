@@ -30,8 +30,9 @@
  * for a fixed descriptor on a fixed device.
  *
  * Supported shapes: D in {4, 8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 512.
- * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation (D = 8 as the lower half of a
- * 16-wide product whose upper half meets zeros; with a single head of width 8, on the CUDA cores).
+ * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation (D = 8 and 4 as part of a 16-wide
+ * product whose other columns meet zeros; tensors of fewer than 16 feature columns, or with D = 4 and an odd
+ * number of heads, on the CUDA cores).
  *
  * Every entry point returns a flare_status_t; nothing is thrown, nothing is printed.
  */

@@ -95,17 +95,17 @@ SimtPlan simt_plan(const flare_desc_t *d, int sms) {
     return p;
 }
 
-// The tensor-core kernels take bfloat16 with D in {16, 32, 64} and a positive scale, and D = 8 with at least two
-// heads as the half-width form of the D = 16 kernels (a token tile of 16 feature columns then spans two heads, so
-// a tensor of one head would be narrower than the tile); everything else (float32, non-positive scale) runs on
-// the CUDA-core kernels.  FLARE_DEBUG_PATH=simt forces the latter.
+// The tensor-core kernels take bfloat16 with D in {16, 32, 64} and a positive scale, and D = 8 or 4 as the narrow
+// forms of the D = 16 kernels: a token tile of 16 feature columns then spans two or four heads, so the tensor must
+// be at least 16 columns wide, and (TMA) its rows a multiple of 16 bytes.  Everything else (float32, non-positive
+// scale, narrower tensors) runs on the CUDA-core kernels.  FLARE_DEBUG_PATH=simt forces the latter.
 bool use_tc(const flare_desc_t *d) {
     static const bool forced_simt = [] {
         const char *e = std::getenv("FLARE_DEBUG_PATH");
         return e != nullptr && std::strcmp(e, "simt") == 0;
     }();
     return !forced_simt && d->dtype == FLARE_DTYPE_BF16 && d->scale > 0.f &&
-           (d->D == 16 || d->D == 32 || d->D == 64 || (d->D == 8 && d->H >= 2));
+           (d->D == 16 || d->D == 32 || d->D == 64 || (d->D == 8 && d->H >= 2) || (d->D == 4 && d->H >= 4 && d->H % 2 == 0));
 }
 
 // Launch plan of the tensor-core encode: `pairs` CTAs per head along the latents (two 128-latent blocks each),
@@ -203,7 +203,7 @@ int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
 constexpr float kLog2e = 1.4426950408889634f;
 
 // kDz: the backward's dZ form of the kernel (V is then dY, lse_dec the decode log-sum-exp rows, pm and pl unused).
-template <int D, bool kPair, bool kDz = false, bool kHalf = false>
+template <int D, bool kPair, bool kDz = false, int DRT = 0>
 int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
                      const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
                      const float *lse_dec = nullptr) {
@@ -212,12 +212,12 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, DG)) != FLARE_OK) return rc;
     if ((rc = make_token_map(&tmV, V, d, kTile, DG)) != FLARE_OK) return rc;
-    if (kHalf) tmQ = tmK;   // unused: the half-width form stages Q with its threads
+    if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = EncodeSmem<DG>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     EncodeTcArgs a;
@@ -228,12 +228,12 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair, kDz, kHalf><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz, DRT><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 
-template <int D, bool kHalf = false>
+template <int D, int DRT = 0>
 int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
                      const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
                      const float *lse_dec, const float *dd, float *part, uint32_t *status, cudaStream_t st) {
@@ -242,12 +242,12 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
     if ((rc = make_token_map(&tmV, V, d, kTile, D)) != FLARE_OK) return rc;
     if ((rc = make_token_map(&tmG, dY, d, kTile, D)) != FLARE_OK) return rc;
-    if (kHalf) tmQ = tmK;   // unused: the half-width form stages Q with its threads
+    if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = BwdDqSmem<D>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_tc_kernel<D, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     BwdDqTcArgs a;
@@ -258,12 +258,12 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, d->H * p.pairs, d->B);
-    bwd_dq_tc_kernel<D, kHalf><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_dq_tc_kernel<D, DRT><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 
-template <int D, bool kHalf = false>
+template <int D, int DRT = 0>
 int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
                         const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
                         const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st) {
@@ -272,7 +272,7 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
     if ((rc = make_token_map(&tmV, V, d, kTile, D)) != FLARE_OK) return rc;
     if ((rc = make_token_map(&tmG, dY, d, kTile, D)) != FLARE_OK) return rc;
-    if (kHalf) tmQ = tmK;   // unused: the half-width form stages Q with its threads
+    if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     BwdTokTcArgs a;
     a.stages = BwdTokSmem<D>::stages(d->M);
@@ -280,7 +280,7 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     const size_t smem = BwdTokSmem<D>::total(a.stages, d->M);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
@@ -292,23 +292,23 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     long per_head = sms / ((long)d->B * d->H);
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
-    bwd_token_tc_kernel<D, kHalf><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_token_tc_kernel<D, DRT><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 
-template <int D, bool kHalf = false>
+template <int D, int DRT = 0>
 int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
                      float *lse_dec, uint32_t *status, cudaStream_t st) {
     CUtensorMap tmK, tmQ;
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
-    if (kHalf) tmQ = tmK;   // unused: the half-width form stages Q with its threads
+    if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = DecodeSmem<D>::total(d->M);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, kHalf>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     DecodeTcArgs a;
@@ -323,7 +323,7 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
     dim3 grid((unsigned)per_head, d->H, d->B);
-    decode_tc_kernel<D, kHalf><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
+    decode_tc_kernel<D, DRT><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -432,13 +432,13 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     FLARE_CUDA(cudaMemsetAsync(ws, 0, kHeaderBytes, st));
     int dz_parts = pa.P;
     bool dz_on_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value && D >= 8) {
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         if (bwd_dz_on_tensor_cores(d)) {
             const TcEncodePlan tp = tc_encode_plan(d, sms);
             uint32_t *status = reinterpret_cast<uint32_t *>(ws);
             int rc;
-            if constexpr (D == 8) {
-                rc = launch_encode_tc<16, false, true, true>(d, tp, Q, K, dY, nullptr, nullptr, nullptr, part, status, st, lse_dec);
+            if constexpr (D < 16) {
+                rc = launch_encode_tc<16, false, true, D>(d, tp, Q, K, dY, nullptr, nullptr, nullptr, part, status, st, lse_dec);
             } else if constexpr (D <= 32) {
                 rc = encode_head_pairs(d)
                          ? launch_encode_tc<D, true, true>(d, tp, Q, K, dY, nullptr, nullptr, nullptr, part, status, st, lse_dec)
@@ -461,10 +461,10 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     bwd_de_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(dZ, Z, de, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
     bool tok_on_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value && D >= 8 && D <= 32) {
-        constexpr int DK = D == 8 ? 16 : D;                     // width the kernels multiply (D = 8: half-width form)
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && D <= 32) {
+        constexpr int DK = D < 16 ? 16 : D;                     // width the kernels multiply (D < 16: narrow forms)
         if (bwd_dq_on_tensor_cores(d) && BwdTokSmem<DK>::stages(d->M) >= 1) {
-            const int rc = launch_bwd_token_tc<DK, D == 8>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd,
+            const int rc = launch_bwd_token_tc<DK, (D < 16 ? D : 0)>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd,
                                                   reinterpret_cast<uint32_t *>(ws), st);
             if (rc != FLARE_OK) return rc;
             tok_on_tc = true;
@@ -478,9 +478,9 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     }
     int dq_parts = pb.P;
     bool dq_on_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value && D >= 8 && D <= 32) {
+    if constexpr (std::is_same<T, __nv_bfloat16>::value && D <= 32) {
         if (bwd_dq_on_tensor_cores(d)) {
-            const int rc = launch_bwd_dq_tc<D == 8 ? 16 : D, D == 8>(d, tc_dq_plan(d, sms), Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part,
+            const int rc = launch_bwd_dq_tc<(D < 16 ? 16 : D), (D < 16 ? D : 0)>(d, tc_dq_plan(d, sms), Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part,
                                                reinterpret_cast<uint32_t *>(ws), st);
             if (rc != FLARE_OK) return rc;
             dq_parts = tc_dq_plan(d, sms).P;
@@ -550,7 +550,8 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
             rc = d->D == 16 ? launch_encode_tc<16, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
                             : launch_encode_tc<32, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
         else
-            rc = d->D == 8    ? launch_encode_tc<16, false, false, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+            rc = d->D == 4    ? launch_encode_tc<16, false, false, 4>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
+                 : d->D == 8  ? launch_encode_tc<16, false, false, 8>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
                  : d->D == 16 ? launch_encode_tc<16, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
                  : d->D == 32 ? launch_encode_tc<32, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
                               : launch_encode_tc<64, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
@@ -570,7 +571,8 @@ int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float
                 uint32_t *status, cudaStream_t st) {
     if (use_tc(d)) {
         const int sms = device_info().sms;
-        return d->D == 8    ? launch_decode_tc<16, true>(d, sms, Q, K, Z, Y, lse_dec, status, st)
+        return d->D == 4    ? launch_decode_tc<16, 4>(d, sms, Q, K, Z, Y, lse_dec, status, st)
+               : d->D == 8  ? launch_decode_tc<16, 8>(d, sms, Q, K, Z, Y, lse_dec, status, st)
                : d->D == 16 ? launch_decode_tc<16>(d, sms, Q, K, Z, Y, lse_dec, status, st)
                : d->D == 32 ? launch_decode_tc<32>(d, sms, Q, K, Z, Y, lse_dec, status, st)
                             : launch_decode_tc<64>(d, sms, Q, K, Z, Y, lse_dec, status, st);

@@ -48,16 +48,17 @@ struct BwdDqSmem {
     }
 };
 
-// grid = (splits, H * pairs, B), as the encode kernel.  kHalf: the half-width form of the forward kernels (the head
-// is DR = D/2 wide in memory; token tiles carry the next head's features in their upper half, every latent
-// operand zeros, and the upper half of the partial dQ is dropped).
-template <int D, bool kHalf = false>
+// grid = (splits, H * pairs, B), as the encode kernel.  DRT = 8 or 4 (with D = 16): the narrow form of the forward
+// kernels (the head is DRT wide in memory; token tiles carry the neighbouring heads' features beside the head's
+// own, every latent operand zeros there, and the other columns of the partial dQ are dropped).
+template <int D, int DRT = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdDqTcArgs a) {
     using G = TileGeom<D>;
     using SM = BwdDqSmem<D>;
-    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
+    constexpr bool kHalf = DRT != 0;
+    constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sT = smem + SM::tile_off;
@@ -106,16 +107,25 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int which = i / (2 * kTile * (G::RB / 16)), rem = i % (2 * kTile * (G::RB / 16));
         if (kHalf || rem / (G::RB / 16) >= rows_here) reinterpret_cast<uint4 *>(smem + SM::lat_off(which))[rem] = make_uint4(0, 0, 0, 0);
     }
+    const int off = kHalf ? narrow_offset(h, DR) : 0;           // the head's first column within a token tile row
     if (kHalf) {
         __syncthreads();
-        for (int i = threadIdx.x; i < rows_here * (DR / 8); i += kTcThreads) {
-            const int m = i / (DR / 8), ch = i % (DR / 8);
-            *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
-                *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
+        if constexpr (DR == 4) {
+            const size_t r0 = ((size_t)b * a.H + h) * M + lb0 * kTile;
+            stage_rows4<D>(sQ, a.Q + ((size_t)h * M + lb0 * kTile) * DR, rows_here, off);
+            stage_rows4_hilo<D>(smem + SM::lat_off(1), smem + SM::lat_off(2), a.Z + r0 * DR, rows_here, off);
+            stage_rows4_hilo<D>(smem + SM::lat_off(3), smem + SM::lat_off(4), a.dZ + r0 * DR, rows_here, off);
+        } else {
+            for (int i = threadIdx.x; i < rows_here * (DR / 8); i += kTcThreads) {
+                const int m = i / (DR / 8), ch = i % (DR / 8);
+                *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
+                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
+            }
         }
     }
-    for (int i = threadIdx.x; i < 2 * rows_here * (DR / 8); i += kTcThreads) {
-        const int which = i / (rows_here * (DR / 8)), rem = i % (rows_here * (DR / 8)), m = rem / (DR / 8), ch = rem % (DR / 8);
+    constexpr int ZC = DR >= 8 ? DR / 8 : 1;                    // 8-float chunks per row (none for DR = 4: staged above)
+    for (int i = threadIdx.x; i < (DR >= 8 ? 2 * rows_here * ZC : 0); i += kTcThreads) {
+        const int which = i / (rows_here * ZC), rem = i % (rows_here * ZC), m = rem / ZC, ch = rem % ZC;
         const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + lb0 * kTile + m) * DR + ch * 8;
         const float4 lo4 = *reinterpret_cast<const float4 *>(src), hi4 = *reinterpret_cast<const float4 *>(src + 4);
         const float z[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
@@ -149,9 +159,9 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / kBqStages) & 1) ^ 1, abort_flag, kErrBwdDq | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(T_FULL + s), 3 * G::TILE_BYTES);
                 uint8_t *dst = sT + (size_t)s * 3 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * DR, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * DR, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -340,10 +350,15 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const long rows = (long)a.B * a.H * M;
             const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);
             float4 *dst = reinterpret_cast<float4 *>(a.part + ((size_t)part * rows + ((size_t)b * a.H + h) * M + m) * DR);
+            if (DR == 4) {
+                dst[0] = make_float4(__uint_as_float(off ? acc[4] : acc[0]), __uint_as_float(off ? acc[5] : acc[1]),
+                                     __uint_as_float(off ? acc[6] : acc[2]), __uint_as_float(off ? acc[7] : acc[3]));
+            } else {
 #pragma unroll
-            for (int dc = 0; dc < DR / 4; ++dc)
-                dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
-                                      __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
+                for (int dc = 0; dc < DR / 4; ++dc)
+                    dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
+                                          __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
+            }
         }
     }
     ptx::tc_fence_before();
@@ -405,8 +420,9 @@ struct BwdTokSmem {
 };
 
 // grid = (CTAs per head, H, B); a CTA takes the token tiles blockIdx.x, blockIdx.x + gridDim.x, ...
-// kHalf: the half-width form (head DR = D/2 wide in memory; the upper halves of the rows of dK and dV are dropped).
-template <int D, bool kHalf = false>
+// DRT = 8 or 4 (with D = 16): the narrow form (head DRT wide in memory; only the head's columns of the rows of dK
+// and dV are kept).
+template <int D, int DRT = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdTokTcArgs a) {
@@ -414,7 +430,8 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     using SM = BwdTokSmem<D>;
     constexpr int UNIT = BwdTokGeom<D>::kUnit;
     constexpr int kMaxSt = BwdTokGeom<D>::kMaxStages;
-    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
+    constexpr bool kHalf = DRT != 0;
+    constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int M = a.M, MU = SM::padded_m(M), stages = a.stages;
@@ -452,12 +469,20 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int which = i / ((MU - zfirst) * (G::RB / 16)), rem = i % ((MU - zfirst) * (G::RB / 16));
         reinterpret_cast<uint4 *>(smem + SM::lat_off(stages, M, which) + (size_t)zfirst * G::RB)[rem] = make_uint4(0, 0, 0, 0);
     }
+    const int off = kHalf ? narrow_offset(h, DR) : 0;           // the head's first column within a token tile row
     if (kHalf) {
         __syncthreads();
-        for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
-            const int m = i / (DR / 8), ch = i % (DR / 8);
-            *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
-                *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + ch * 8);
+        if constexpr (DR == 4) {
+            const size_t r0 = ((size_t)b * a.H + h) * M;
+            stage_rows4<D>(sQ, a.Q + (size_t)h * M * DR, M, off);
+            stage_rows4_hilo<D>(smem + SM::lat_off(stages, M, 1), smem + SM::lat_off(stages, M, 2), a.Z + r0 * DR, M, off);
+            stage_rows4_hilo<D>(smem + SM::lat_off(stages, M, 3), smem + SM::lat_off(stages, M, 4), a.dZ + r0 * DR, M, off);
+        } else {
+            for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+                const int m = i / (DR / 8), ch = i % (DR / 8);
+                *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
+                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + ch * 8);
+            }
         }
     }
     for (int m = threadIdx.x; m < MU; m += kTcThreads) {
@@ -471,8 +496,9 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         cst[m] = nle;
         cst[MU + m] = nde;
     }
-    for (int i = threadIdx.x; i < 2 * M * (DR / 8); i += kTcThreads) {
-        const int which = i / (M * (DR / 8)), rem = i % (M * (DR / 8)), m = rem / (DR / 8), ch = rem % (DR / 8);
+    constexpr int ZC = DR >= 8 ? DR / 8 : 1;                    // 8-float chunks per row (none for DR = 4: staged above)
+    for (int i = threadIdx.x; i < (DR >= 8 ? 2 * M * ZC : 0); i += kTcThreads) {
+        const int which = i / (M * ZC), rem = i % (M * ZC), m = rem / ZC, ch = rem % ZC;
         const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + m) * DR + ch * 8;
         const float4 lo4 = *reinterpret_cast<const float4 *>(src), hi4 = *reinterpret_cast<const float4 *>(src + 4);
         const float z[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
@@ -506,9 +532,9 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / stages) & 1) ^ 1, abort_flag, kErrBwdTok | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(T_FULL + s), 3 * G::TILE_BYTES);
                 uint8_t *dst = smem + (size_t)s * 3 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR, t * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * DR, t * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * DR, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR - off, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(T_FULL + s), h * DR - off, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + 2 * G::TILE_BYTES), &tmG, bar(T_FULL + s), h * DR - off, t * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -610,6 +636,12 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             if (p_inside) {
                 a.dd[p_ddi] = p_dd;
                 uint4 *dk = reinterpret_cast<uint4 *>(a.dK + p_tok * DR), *dv = reinterpret_cast<uint4 *>(a.dV + p_tok * DR);
+                if (DR == 4) {
+                    auto k4 = [&](int i) { return __uint_as_float(off ? ak[4 + i] : ak[i]) * a.scale; };
+                    auto v4 = [&](int i) { return __uint_as_float(off ? avv[4 + i] : avv[i]); };
+                    *reinterpret_cast<uint2 *>(dk) = make_uint2(ptx::pack_bf16(k4(0), k4(1)), ptx::pack_bf16(k4(2), k4(3)));
+                    *reinterpret_cast<uint2 *>(dv) = make_uint2(ptx::pack_bf16(v4(0), v4(1)), ptx::pack_bf16(v4(2), v4(3)));
+                }
 #pragma unroll
                 for (int q = 0; q < DR / 8; ++q) {
                     uint32_t wk[4], wv4[4];

@@ -57,6 +57,37 @@ struct TileGeom {
     __device__ static __forceinline__ int swz(int r) { return RB == 32 ? ((r >> 2) & 1) : RB == 64 ? ((r >> 1) & 3) : (r & 7); }
 };
 
+// Narrow heads (half- and quarter-width forms of the kernels): the head is DR < D wide in memory and the kernels
+// multiply D = 16 wide rows.  A token tile is the 16 feature columns from the 16-byte boundary at or below the
+// head's first column (a TMA box must start on one), so the head's features sit `off` elements into the row
+// (0, or 4 for every other head of width 4) next to its neighbours' (zeros past the last head).  The rows of the
+// latent operands (Q, Z, dZ) are staged by the CTA's threads into zeroed rows at the same offset, so the
+// neighbours' columns meet zeros in every product; accumulator columns outside [off, off + DR) are never read.
+__device__ __forceinline__ int narrow_offset(int h, int DR) { return (h * DR) & 7; }
+
+// rows of a [rows, 4] bf16 matrix -> columns [off, off + 4) of zeroed, swizzled D-wide rows
+template <int D>
+__device__ __forceinline__ void stage_rows4(uint8_t *dst, const __nv_bfloat16 *src, int rows, int off) {
+    using G = TileGeom<D>;
+    for (int m = threadIdx.x; m < rows; m += blockDim.x)
+        *reinterpret_cast<uint2 *>(dst + (size_t)m * G::RB + (G::swz(m) << 4) + off * 2) =
+            *reinterpret_cast<const uint2 *>(src + (size_t)m * 4);
+}
+// rows of a [rows, 4] float matrix -> two bf16 halves (hi = round(z), lo = round(z - hi)) at columns [off, off + 4)
+template <int D>
+__device__ __forceinline__ void stage_rows4_hilo(uint8_t *dst_hi, uint8_t *dst_lo, const float *src, int rows, int off) {
+    using G = TileGeom<D>;
+    for (int m = threadIdx.x; m < rows; m += blockDim.x) {
+        const float4 z = *reinterpret_cast<const float4 *>(src + (size_t)m * 4);
+        const uint32_t h0 = ptx::pack_bf16(z.x, z.y), h1 = ptx::pack_bf16(z.z, z.w);
+        const uint32_t l0 = ptx::pack_bf16(z.x - __uint_as_float(h0 << 16), z.y - __uint_as_float(h0 & 0xffff0000u));
+        const uint32_t l1 = ptx::pack_bf16(z.z - __uint_as_float(h1 << 16), z.w - __uint_as_float(h1 & 0xffff0000u));
+        const size_t o = (size_t)m * G::RB + (G::swz(m) << 4) + off * 2;
+        *reinterpret_cast<uint2 *>(dst_hi + o) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2 *>(dst_lo + o) = make_uint2(l0, l1);
+    }
+}
+
 // ------------------------------------------------------------------------------------- softmax arithmetic
 // p = 2^(s * sl2 + neg[k]) with one addend per column (read from shared memory, four at a time): the form the
 // backward needs, where every column (token) carries its own log-sum-exp.  The weights leave as two bf16 halves,
@@ -214,14 +245,13 @@ struct DecodeSmem {
 // Decode.  grid = (ctas_per_head, H, B); each CTA walks a contiguous range of 128-token tiles of one (b, h)
 // with Q_h and Z_bh resident in shared memory.
 //
-// Half-width form (kHalf): the head is DR = D/2 wide in memory.  The kernel still multiplies D-wide rows: a token
-// row of the K tile is the head's DR features followed by the next head's (or zeros past the last head), the rows
-// of Q and Z are staged with zeros in their upper half, so the neighbour's features meet zeros in every product.
-// This is how a head width of 8 (the smallest MMA K-step is 16) runs on the tensor cores.
-template <int D, bool kHalf = false>
+// Narrow form (DRT = 8 or 4 with D = 16): the head is DRT wide in memory (see narrow_offset).  This is how head
+// widths below the smallest MMA K-step (16) run on the tensor cores.
+template <int D, int DRT = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
-    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
+    constexpr bool kHalf = DRT != 0;
+    constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     using G = TileGeom<D>;
     using SM = DecodeSmem<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -244,6 +274,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.y, b = blockIdx.z;
+    const int off = kHalf ? narrow_offset(h, DR) : 0;           // the head's first column within a token tile row
     const int t_begin = (int)((long)a.tiles * blockIdx.x / gridDim.x);
     const int t_end = (int)((long)a.tiles * (blockIdx.x + 1) / gridDim.x);
     const int ntiles = t_end - t_begin;
@@ -283,14 +314,20 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 reinterpret_cast<uint4 *>(sZ + (size_t)M * G::RB)[i] = make_uint4(0, 0, 0, 0);
             }
             __syncthreads();
-            for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
-                const int m = i / (DR / 8), c = i % (DR / 8);
-                *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) =
-                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + c * 8);
+            if constexpr (DR == 4) {
+                stage_rows4<D>(sQ, a.Q + (size_t)h * M * DR, M, off);
+                stage_rows4_hilo<D>(sZ, sZ + (size_t)M * G::RB, Zg, M, off);
+            } else {
+                for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+                    const int m = i / (DR / 8), c = i % (DR / 8);
+                    *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) =
+                        *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + c * 8);
+                }
             }
         }
-        for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
-            const int m = i / (DR / 8), c = i % (DR / 8);
+        constexpr int ZC = DR >= 8 ? DR / 8 : 1;                // 8-float chunks per row of Z (none for DR = 4: staged above)
+        for (int i = threadIdx.x; i < (DR >= 8 ? M * ZC : 0); i += kTcThreads) {
+            const int m = i / ZC, c = i % ZC;
             const float4 lo = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8);
             const float4 hi = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8 + 4);
             const float z[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
@@ -327,7 +364,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int s = i % nstages;
                 if (!ptx::mbar_wait(bar(K_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrDecode | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(K_FULL + s), G::TILE_BYTES);
-                ptx::tma_load_3d(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), &tmK, bar(K_FULL + s), h * DR,
+                ptx::tma_load_3d(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), &tmK, bar(K_FULL + s), h * DR - off,
                                  (t_begin + i) * kTile, b);
             }
         }
@@ -495,7 +532,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                 }
-                if (n < a.N) {
+                if (DR == 4) {
+                    if (n < a.N)
+                        *reinterpret_cast<uint2 *>(dst) =
+                            make_uint2(ptx::pack_bf16((off ? y[4] : y[0]) * inv, (off ? y[5] : y[1]) * inv),
+                                       ptx::pack_bf16((off ? y[6] : y[2]) * inv, (off ? y[7] : y[3]) * inv));
+                } else if (n < a.N) {
                     dst[2 * dc] = make_uint4(ptx::pack_bf16(y[0] * inv, y[1] * inv), ptx::pack_bf16(y[2] * inv, y[3] * inv),
                                              ptx::pack_bf16(y[4] * inv, y[5] * inv), ptx::pack_bf16(y[6] * inv, y[7] * inv));
                     if (DR > 8 + 16 * dc)
@@ -571,16 +613,17 @@ struct EncodeSmem {
 // and the weights are already normalised, so there is no running maximum, no rescaling and no sum; tokens
 // beyond N get the shift -inf.  Every group leaves one partial sum of dZ per split (part_acc).
 //
-// Half-width form (kHalf; not with kPair): the head is DR = D/2 wide in memory, as in the decode kernel: K and V
-// tile rows carry the next head's features in their upper half, Q rows zeros; the upper half of the accumulator
-// (weights times the neighbour's values) is dropped.
-template <int D, bool kPair, bool kDz = false, bool kHalf = false>
+// Narrow form (DRT = 8 or 4 with D = 16; not with kPair): the head is DRT wide in memory, as in the decode kernel:
+// K and V tile rows carry the neighbouring heads' features beside the head's own, Q rows zeros there; accumulator
+// columns outside the head's (weights times the neighbours' values) are dropped.
+template <int D, bool kPair, bool kDz = false, int DRT = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
-    static_assert(!(kPair && kHalf), "head pairing and the half-width form exclude each other");
+    constexpr bool kHalf = DRT != 0;
+    static_assert(!(kPair && kHalf), "head pairing and the narrow form exclude each other");
     constexpr int DG = kPair ? 2 * D : D;
-    constexpr int DR = kHalf ? D / 2 : D;                       // head width in memory
+    constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     using G = TileGeom<DG>;
     using SM = EncodeSmem<DG>;
     extern __shared__ uint8_t smem_raw[];
@@ -609,6 +652,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
     const int rows_q = min(M - lb0 * kTile, 2 * kTile);                  // latent rows of this CTA
+    const int off = kHalf ? narrow_offset(h, DR) : 0;                    // the head's first column within a tile row
     const int rows_here = (kPair || kHalf) ? 0 : rows_q;                 // ... fetched by TMA
     constexpr int SLOT_COLS = 256;   // per slot and half (128 columns): two score buffers of UNIT columns, accumulator at 64
     constexpr int HALF = kTile / 2;
@@ -646,10 +690,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (kHalf) {
         // rows [Q[h][m] | 0]: the lower DR/8 chunks of every row, the rest stays zero
         __syncthreads();
-        for (int i = threadIdx.x; i < rows_q * (DR / 8); i += kTcThreads) {
-            const int m = i / (DR / 8), ch = i % (DR / 8);
-            *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
-                *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
+        if constexpr (DR == 4) {
+            stage_rows4<DG>(sQ, a.Q + ((size_t)h * M + lb0 * kTile) * DR, rows_q, off);
+        } else {
+            for (int i = threadIdx.x; i < rows_q * (DR / 8); i += kTcThreads) {
+                const int m = i / (DR / 8), ch = i % (DR / 8);
+                *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
+                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
+            }
         }
     }
     ptx::fence_proxy_async_smem();
@@ -672,8 +720,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (!ptx::mbar_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(KV_FULL + s), 2 * G::TILE_BYTES);
                 uint8_t *dst = sKV + (size_t)s * 2 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(KV_FULL + s), h * DR, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(KV_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -856,10 +904,15 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 a.part_l[prow] = l2.x + l2.y;
             }
             float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * DR);
+            if (DR == 4) {
+                dst[0] = make_float4(__uint_as_float(off ? acc[4] : acc[0]), __uint_as_float(off ? acc[5] : acc[1]),
+                                     __uint_as_float(off ? acc[6] : acc[2]), __uint_as_float(off ? acc[7] : acc[3]));
+            } else {
 #pragma unroll
-            for (int dc = 0; dc < DR / 4; ++dc)
-                dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
-                                      __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
+                for (int dc = 0; dc < DR / 4; ++dc)
+                    dst[dc] = make_float4(__uint_as_float(acc[4 * dc]), __uint_as_float(acc[4 * dc + 1]),
+                                          __uint_as_float(acc[4 * dc + 2]), __uint_as_float(acc[4 * dc + 3]));
+            }
         }
     }
     ptx::tc_fence_before();

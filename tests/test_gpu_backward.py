@@ -92,6 +92,7 @@ EDGE = [
     # head width 4
     (2, 4, 300, 32, 4, "bf16", 0.1),
     (1, 16, 500, 64, 4, "bf16", 0.0),
+    (12, 16, 500, 144, 4, "bf16", 0.2),
     (1, 2, 200, 7, 4, "f32", 0.0),
 ]
 

@@ -57,6 +57,8 @@ EDGE = [
     # head width 4 (the paper's other setting for its PDE models)
     (2, 4, 300, 32, 4, "bf16", 0.1),
     (1, 16, 700, 64, 4, "bf16", 0.0),
+    (12, 16, 500, 144, 4, "bf16", 0.2),
+    (1, 2, 300, 32, 4, "bf16", 0.0),       # two heads of width 4: narrower than a tile, CUDA cores
     (1, 2, 200, 7, 4, "f32", 0.0),
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 2049, 300, 64, "f32", 0.0),
