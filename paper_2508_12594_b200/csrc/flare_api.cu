@@ -500,9 +500,8 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
             d->N, d->M, pb.LM, pb.chunk, d->scale);
         FLARE_CUDA(cudaGetLastError());
     }
-    const long per_batch = (long)d->H * d->M * d->D;
-    bwd_dq_reduce_kernel<<<(unsigned)((per_batch + 255) / 256), 256, 0, st>>>(part, dQ, dq_parts, d->B, d->H, d->M, d->D,
-                                                                             d->scale);
+    bwd_dq_reduce_kernel<<<(unsigned)((long)d->H * d->M), kDqReduceThreads, 0, st>>>(part, dQ, dq_parts, d->B, d->H, d->M,
+                                                                                     d->D, d->scale);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -561,8 +560,10 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
                                            : launch_encode_simt<__nv_bfloat16>(d, p, Q, K, V, mask, pm, pl, pacc, st);
     }
     if (rc != FLARE_OK) return rc;
-    const long total = rows * d->D;
-    merge_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(pm, pl, pacc, Z, lse_enc, P, rows, d->D);
+    if (P > 8)   // many partials (small problems spread over all SMs): a block per row shares the loads
+        merge_kernel<<<(unsigned)rows, kMergeThreads, 0, st>>>(pm, pl, pacc, Z, lse_enc, P, rows, d->D);
+    else
+        merge_serial_kernel<<<(unsigned)((rows * d->D + 255) / 256), 256, 0, st>>>(pm, pl, pacc, Z, lse_enc, P, rows, d->D);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }

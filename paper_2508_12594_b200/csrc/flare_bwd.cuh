@@ -14,7 +14,7 @@
 //            dQ_m   = scale * sum_b sum_n dS[m,n] k_n                                     (split over N, then summed)
 // dd[n] is formed from the float32 dot products dY_n . Z_m rather than from the stored Y: Y has been rounded to
 // the output type, and where the rows Z_m that a token mixes are nearly equal that rounding would dominate dS.
-// Reductions add their partial results in index order, so the gradients are bitwise reproducible.
+// Reductions add their partial results in a fixed order, so the gradients are bitwise reproducible.
 #pragma once
 
 #include "flare_common.cuh"
@@ -280,18 +280,28 @@ bwd_dq_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
     }
 }
 
-// dQ[h][m][d] = scale * sum_b sum_p part[p][(b,h,m)][d].  One thread per output element.
-__global__ void __launch_bounds__(256)
+// dQ[h][m][d] = scale * sum_b sum_p part[p][(b,h,m)][d].  One block per (h, m): thread (slice, d) adds the terms
+// q = b * P + p with q = slice, slice + S, ... (S = 128 / D) in index order, thread (0, d) the S slice sums in index
+// order: a fixed order, and the B * P loads of a row are spread over the block.
+constexpr int kDqReduceThreads = 128;
+__global__ void __launch_bounds__(kDqReduceThreads)
 bwd_dq_reduce_kernel(const float *__restrict__ part, float *__restrict__ dQ, int P, int B, int H, int M, int D,
                      float scale) {
-    const long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long per_batch = (long)H * M * D;
-    if (idx >= per_batch) return;
-    const long rows = (long)B * H * M;
+    __shared__ float s_a[kDqReduceThreads];
+    const long hm = blockIdx.x;                                  // h * M + m
+    const int t = threadIdx.x, S = kDqReduceThreads / D, d = t % D, slice = t / D;
+    const long per_batch = (long)H * M, rows = (long)B * per_batch;
     float s = 0.f;
-    for (int b = 0; b < B; ++b)
-        for (int p = 0; p < P; ++p) s += part[(size_t)p * rows * D + (size_t)b * per_batch + idx];
-    dQ[idx] = s * scale;
+    for (int q = slice; q < B * P; q += S) {
+        const int b = q / P, p = q % P;
+        s += part[((size_t)p * rows + (size_t)b * per_batch + hm) * D + d];
+    }
+    s_a[t] = s;
+    __syncthreads();
+    if (slice == 0) {
+        for (int k = 1; k < S; ++k) s += s_a[k * D + d];
+        dQ[hm * D + d] = s * scale;
+    }
 }
 
 }  // namespace flare

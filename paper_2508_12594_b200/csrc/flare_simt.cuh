@@ -101,10 +101,55 @@ encode_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
 
 // Log-sum-exp merge of the P partial results of every latent row (b, h, m):
 //   m* = max_p m_p;  l = sum_p l_p exp(m_p - m*);  Z = sum_p acc_p exp(m_p - m*) / l;  lse = m* + log l.
-// One thread per (row, d); partials are added in index order, so the result is reproducible.
-__global__ void __launch_bounds__(256)
+// One block per row: thread (slice, d) adds the partials p = slice, slice + S, ... (S = 128 / D slices) in index
+// order, thread (0, d) then adds the S slice sums in index order: a fixed order, so the result is reproducible,
+// and the P loads of a row are spread over the block instead of queued in one thread (with P in the hundreds
+// for small problems the serial form took longer than the encode kernel itself).
+constexpr int kMergeThreads = 128;
+__global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const float *__restrict__ part_m, const float *__restrict__ part_l, const float *__restrict__ part_acc,
              float *__restrict__ Z, float *__restrict__ lse_enc, int P, long rows, int D) {
+    __shared__ float s_a[kMergeThreads], s_b[kMergeThreads];
+    const long row = blockIdx.x;
+    const int t = threadIdx.x, S = kMergeThreads / D, d = t % D, slice = t / D;
+    float mx = -INFINITY;
+    for (int p = t; p < P; p += kMergeThreads) mx = fmaxf(mx, part_m[(size_t)p * rows + row]);
+    s_a[t] = mx;
+    __syncthreads();
+    for (int w = kMergeThreads / 2; w > 0; w >>= 1) {
+        if (t < w) s_a[t] = fmaxf(s_a[t], s_a[t + w]);
+        __syncthreads();
+    }
+    const float mstar = s_a[0];
+    __syncthreads();
+    if (mstar == -INFINITY) {  // no valid token anywhere
+        if (t < D) Z[row * D + t] = 0.f;
+        if (lse_enc != nullptr && t == 0) lse_enc[row] = -INFINITY;
+        return;
+    }
+    float l = 0.f, z = 0.f;
+    for (int p = slice; p < P; p += S) {
+        const float w = expf(part_m[(size_t)p * rows + row] - mstar);
+        l = fmaf(part_l[(size_t)p * rows + row], w, l);
+        z = fmaf(part_acc[((size_t)p * rows + row) * D + d], w, z);
+    }
+    s_a[t] = l;
+    s_b[t] = z;
+    __syncthreads();
+    if (slice == 0) {
+        for (int k = 1; k < S; ++k) {
+            l += s_a[k * D + d];
+            z += s_b[k * D + d];
+        }
+        Z[row * D + d] = z / l;
+        if (lse_enc != nullptr && d == 0) lse_enc[row] = mstar + logf(l);
+    }
+}
+
+// The same merge with one thread per (row, d), partials added in index order: for few partials and many rows.
+__global__ void __launch_bounds__(256)
+merge_serial_kernel(const float *__restrict__ part_m, const float *__restrict__ part_l, const float *__restrict__ part_acc,
+                    float *__restrict__ Z, float *__restrict__ lse_enc, int P, long rows, int D) {
     const long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * D) return;
     const long row = idx / D;
