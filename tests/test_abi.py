@@ -64,6 +64,16 @@ def test_descriptor_validation_needs_no_device(lib):
     assert rc == flare.ERR_UNSUPPORTED
 
 
+def test_every_head_width_of_the_paper_is_accepted(lib):
+    """D = 4 and 8 (the paper's PDE models: C = 64 with 16 or 8 heads) up to 64, both dtypes, all operations."""
+    for D in (4, 8, 16, 32, 64):
+        for dtype in (flare.DTYPE_F32, flare.DTYPE_BF16):
+            desc = flare.FlareDesc(2, 64 // D if D <= 16 else 2, 1000, 64, D, dtype, 1.0)
+            for op in (flare.OP_ENCODE, flare.OP_FORWARD, flare.OP_BACKWARD):
+                assert flare.flare_workspace_bytes(desc, op) > 0, (D, dtype, op)
+    assert flare.flare_workspace_bytes(flare.FlareDesc(2, 4, 1000, 64, 2, flare.DTYPE_BF16, 1.0), flare.OP_FORWARD) == 0
+
+
 def test_workspace_never_scales_with_n_times_m(lib):
     """Scratch is O(partials * B*H*M*(D+2)): growing N a thousandfold must not grow it by the same factor."""
     small = flare.FlareDesc(1, 8, 4096, 256, 16, flare.DTYPE_BF16, 1.0)
