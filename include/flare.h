@@ -29,7 +29,7 @@
  * run concurrently on different streams only with different workspaces.  Results are bitwise reproducible
  * for a fixed descriptor on a fixed device.
  *
- * Supported shapes: D in {4, 8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 512.
+ * Supported shapes: D in {4, 8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 2048.
  * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation (D = 8 and 4 as part of a 16-wide
  * product whose other columns meet zeros; tensors of fewer than 16 feature columns, or with D = 4 and an odd
  * number of heads, on the CUDA cores).

@@ -68,7 +68,7 @@ int check_desc(const flare_desc_t *d) {
     if (!std::isfinite(d->scale)) return FLARE_ERR_INVALID_ARG;
     if (d->dtype != FLARE_DTYPE_F32 && d->dtype != FLARE_DTYPE_BF16) return FLARE_ERR_UNSUPPORTED;
     if (d->D != 4 && d->D != 8 && d->D != 16 && d->D != 32 && d->D != 64) return FLARE_ERR_UNSUPPORTED;
-    if (d->dtype == FLARE_DTYPE_BF16 && (d->M % 16 != 0 || d->M < 16 || d->M > 512)) return FLARE_ERR_UNSUPPORTED;
+    if (d->dtype == FLARE_DTYPE_BF16 && (d->M % 16 != 0 || d->M < 16 || d->M > 2048)) return FLARE_ERR_UNSUPPORTED;
     if ((long)d->B * d->N > (1L << 31) - 1 || d->H > 65535 || d->B > 65535) return FLARE_ERR_UNSUPPORTED;
     return FLARE_OK;
 }
@@ -568,9 +568,13 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
     return FLARE_OK;
 }
 
+// One decode launch holds all M score columns of a token tile in tensor memory (512 columns) and Q_h, Z_h in shared
+// memory: up to kDecodeMaxM latents.
+constexpr int kDecodeMaxM = 512;
+
 int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
                 uint32_t *status, cudaStream_t st) {
-    if (use_tc(d)) {
+    if (use_tc(d) && d->M <= kDecodeMaxM) {
         const int sms = device_info().sms;
         return d->D == 4    ? launch_decode_tc<16, 4>(d, sms, Q, K, Z, Y, lse_dec, status, st)
                : d->D == 8  ? launch_decode_tc<16, 8>(d, sms, Q, K, Z, Y, lse_dec, status, st)

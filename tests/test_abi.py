@@ -54,7 +54,7 @@ def test_descriptor_validation_needs_no_device(lib):
     assert flare.flare_workspace_bytes(ok, flare.OP_FORWARD) > 0
     assert flare.flare_encode_partials(ok) >= 1
     for bad in (flare.FlareDesc(0, 2, 8, 16, 16, 0, 1.0), flare.FlareDesc(1, 2, 8, 16, 12, 0, 1.0),
-                flare.FlareDesc(1, 2, 8, 17, 16, flare.DTYPE_BF16, 1.0), flare.FlareDesc(1, 2, 8, 1024, 16, 1, 1.0),
+                flare.FlareDesc(1, 2, 8, 17, 16, flare.DTYPE_BF16, 1.0), flare.FlareDesc(1, 2, 8, 4096, 16, 1, 1.0),
                 flare.FlareDesc(1, 2, 8, 16, 16, 7, 1.0), flare.FlareDesc(1, 2, 8, 16, 16, 0, float("nan"))):
         assert flare.flare_workspace_bytes(bad, flare.OP_FORWARD) == 0
     # null pointers are rejected before anything touches a device

@@ -60,6 +60,10 @@ EDGE = [
     (12, 16, 500, 144, 4, "bf16", 0.2),
     (1, 2, 300, 32, 4, "bf16", 0.0),       # two heads of width 4: narrower than a tile, CUDA cores
     (1, 2, 200, 7, 4, "f32", 0.0),
+    # more than 512 latents (the paper's million-point study goes to 2048)
+    (1, 2, 700, 1024, 16, "bf16", 0.0),
+    (1, 2, 300, 2048, 8, "bf16", 0.1),
+    (2, 1, 400, 640, 32, "bf16", 0.0),
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 2049, 300, 64, "f32", 0.0),
     (1, 4, 64, 1, 16, "f32", 0.0),
