@@ -80,6 +80,8 @@ const char *flare_last_cuda_error(void);
  * Bytes of scratch `workspace` the given operation needs for `desc` on the current device (0 for an invalid
  * or unsupported descriptor).  Encode writes per-split partial results (running maximum, sum and
  * un-normalised latent rows) there: O(splits * B * H * M * (D + 2)) floats, never anything of size N x M.
+ * The forward over more than 512 bfloat16 latents decodes them in ranges of 512 and adds one float32 row and
+ * one log-sum-exp per token, head and range: ceil(M / 512) * B * N * H * (D + 1) floats.
  */
 size_t flare_workspace_bytes(const flare_desc_t *desc, int op);
 
@@ -97,7 +99,8 @@ int flare_encode(const flare_desc_t *desc, const void *Q_lat, const void *K, con
 
 /*
  * Decode (Section 3.2, decode equation; per-token sum of the design-principles appendix):
- * Y and, if lse_dec != NULL, lse_dec, from K, Q_lat and a latent sequence Z.  Needs no workspace.
+ * Y and, if lse_dec != NULL, lse_dec, from K, Q_lat and a latent sequence Z.  Needs no workspace (and therefore
+ * runs more than 512 bfloat16 latents on the CUDA cores; flare_forward, which has a workspace, does not).
  */
 int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *Z, void *Y,
                  float *lse_dec, flare_stream_t stream);

@@ -299,13 +299,14 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
 
 template <int D, int DRT = 0>
 int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
-                     float *lse_dec, uint32_t *status, cudaStream_t st) {
+                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0 = 0, int mc = 0, float *Ypart = nullptr) {
+    if (mc == 0) mc = d->M;                                     // the launch's range of latents: [m0, m0 + mc)
     CUtensorMap tmK, tmQ;
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
-    const size_t smem = DecodeSmem<D>::total(d->M);
+    const size_t smem = DecodeSmem<D>::total(mc);
     static bool attr_set = false;
     if (!attr_set) {
         FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
@@ -314,10 +315,11 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     DecodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.Y = (__nv_bfloat16 *)Y; a.lse_dec = lse_dec; a.status = status;
-    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = mc;
+    a.mtot = d->M; a.m0 = m0; a.Ypart = Ypart;
     a.sl2 = d->scale * kLog2e;
     a.tiles = (d->N + kTile - 1) / kTile;
-    a.plan = make_decode_plan(d->M, D);
+    a.plan = make_decode_plan(mc, D);
     if (a.plan.cs == 0) return FLARE_ERR_UNSUPPORTED;
     long per_head = sms / ((long)d->B * d->H);
     if (per_head < 1) per_head = 1;
@@ -572,15 +574,49 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
 // memory: up to kDecodeMaxM latents.
 constexpr int kDecodeMaxM = 512;
 
+// Ranges of latents a decode over more than kDecodeMaxM latents is cut into, and the scratch their partial results
+// take after the encode layout of the forward workspace: float32 rows [C][B*N*H][D] and log-sum-exps [C][B*N*H].
+int decode_ranges(const flare_desc_t *d) { return (d->M + kDecodeMaxM - 1) / kDecodeMaxM; }
+bool decode_in_ranges(const flare_desc_t *d) { return use_tc(d) && d->M > kDecodeMaxM; }
+size_t decode_range_bytes(const flare_desc_t *d) {
+    if (!decode_in_ranges(d)) return 0;
+    const size_t rows = (size_t)d->B * d->N * d->H;
+    return align_up(sizeof(float) * decode_ranges(d) * rows * d->D) + align_up(sizeof(float) * decode_ranges(d) * rows);
+}
+
+template <int D, int DRT>
+int decode_tc_any(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
+                  uint32_t *status, char *range_scratch, cudaStream_t st) {
+    if (d->M <= kDecodeMaxM) return launch_decode_tc<D, DRT>(d, sms, Q, K, Z, Y, lse_dec, status, st);
+    constexpr int DR = DRT ? DRT : D;
+    const int C = decode_ranges(d);
+    const size_t rows = (size_t)d->B * d->N * d->H;
+    float *Ypart = reinterpret_cast<float *>(range_scratch);
+    float *lpart = reinterpret_cast<float *>(range_scratch + align_up(sizeof(float) * C * rows * d->D));
+    for (int c = 0; c < C; ++c) {
+        const int m0 = c * kDecodeMaxM, mc = d->M - m0 < kDecodeMaxM ? d->M - m0 : kDecodeMaxM;
+        const int rc = launch_decode_tc<D, DRT>(d, sms, Q, K, Z, nullptr, lpart + (size_t)c * rows, status, st, m0, mc,
+                                                Ypart + (size_t)c * rows * DR);
+        if (rc != FLARE_OK) return rc;
+    }
+    decode_combine_kernel<DR><<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(Ypart, lpart, C, (long)rows,
+                                                                             (__nv_bfloat16 *)Y, lse_dec);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+// range_scratch: decode_range_bytes(d) bytes, or null (then more than kDecodeMaxM latents take the CUDA-core kernel)
 int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
-                uint32_t *status, cudaStream_t st) {
-    if (use_tc(d) && d->M <= kDecodeMaxM) {
+                uint32_t *status, cudaStream_t st, char *range_scratch = nullptr) {
+    if (use_tc(d) && (d->M <= kDecodeMaxM || range_scratch != nullptr)) {
         const int sms = device_info().sms;
-        return d->D == 4    ? launch_decode_tc<16, 4>(d, sms, Q, K, Z, Y, lse_dec, status, st)
-               : d->D == 8  ? launch_decode_tc<16, 8>(d, sms, Q, K, Z, Y, lse_dec, status, st)
-               : d->D == 16 ? launch_decode_tc<16>(d, sms, Q, K, Z, Y, lse_dec, status, st)
-               : d->D == 32 ? launch_decode_tc<32>(d, sms, Q, K, Z, Y, lse_dec, status, st)
-                            : launch_decode_tc<64>(d, sms, Q, K, Z, Y, lse_dec, status, st);
+        switch (d->D) {
+            case 4: return decode_tc_any<16, 4>(d, sms, Q, K, Z, Y, lse_dec, status, range_scratch, st);
+            case 8: return decode_tc_any<16, 8>(d, sms, Q, K, Z, Y, lse_dec, status, range_scratch, st);
+            case 16: return decode_tc_any<16, 0>(d, sms, Q, K, Z, Y, lse_dec, status, range_scratch, st);
+            case 32: return decode_tc_any<32, 0>(d, sms, Q, K, Z, Y, lse_dec, status, range_scratch, st);
+            default: return decode_tc_any<64, 0>(d, sms, Q, K, Z, Y, lse_dec, status, range_scratch, st);
+        }
     }
     return (d->dtype == FLARE_DTYPE_F32) ? launch_decode_simt<float>(d, Q, K, Z, Y, lse_dec, st)
                                          : launch_decode_simt<__nv_bfloat16>(d, Q, K, Z, Y, lse_dec, st);
@@ -641,7 +677,8 @@ size_t flare_workspace_bytes(const flare_desc_t *desc, int op) {
     switch (op) {
         case FLARE_OP_ENCODE: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, false).total;
         case FLARE_OP_DECODE: return kHeaderBytes;
-        case FLARE_OP_FORWARD: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, true).total;
+        case FLARE_OP_FORWARD:
+            return make_layout(partials_for(desc, device_info().sms), rows, desc->D, true).total + decode_range_bytes(desc);
         case FLARE_OP_BACKWARD: return bwd_layout(desc, device_info().sms).total;
         default: return 0;
     }
@@ -702,14 +739,13 @@ int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, co
         return FLARE_ERR_INVALID_ARG;
     if ((rc = require_device()) != FLARE_OK) return rc;
     if (workspace_bytes < flare_workspace_bytes(desc, FLARE_OP_FORWARD)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
-    if (Z == nullptr) {
-        const long rows = (long)desc->B * desc->H * desc->M;
-        WorkspaceLayout w = make_layout(partials_for(desc, device_info().sms), rows, desc->D, true);
-        Z = reinterpret_cast<float *>(static_cast<char *>(workspace) + w.z);
-    }
+    const WorkspaceLayout w = make_layout(partials_for(desc, device_info().sms), (long)desc->B * desc->H * desc->M, desc->D, true);
+    if (Z == nullptr) Z = reinterpret_cast<float *>(static_cast<char *>(workspace) + w.z);
     rc = encode_impl(desc, Q_lat, K, V, key_mask, Z, lse_enc, workspace, (cudaStream_t)stream);
     if (rc != FLARE_OK) return rc;
-    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, reinterpret_cast<uint32_t *>(workspace), (cudaStream_t)stream);
+    char *range_scratch = decode_in_ranges(desc) ? static_cast<char *>(workspace) + w.total : nullptr;
+    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, reinterpret_cast<uint32_t *>(workspace), (cudaStream_t)stream,
+                       range_scratch);
 }
 
 int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,

@@ -212,7 +212,10 @@ struct DecodeTcArgs {
     __nv_bfloat16 *Y;    // [B,N,H,D]
     float *lse_dec;      // [B,N,H] or null
     uint32_t *status;    // workspace header or null
-    int B, H, N, M;
+    int B, H, N, M;      // M: latents this launch works on (all of them, or a range of at most 512)
+    int mtot, m0;        // latents per head in Q and Z, and the first one of this launch's range
+    float *Ypart;        // null, or [B,N,H,D] float32: rows normalised over the range go here instead of Y, with
+                         // their log-sum-exp in lse_dec, for decode_combine_kernel
     float sl2;           // scale * log2(e)
     int tiles;           // ceil(N / 128)
     DecodePlan plan;
@@ -306,7 +309,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // Z_bh -> two bf16 halves (hi = round(z), lo = round(z - hi)); rows of RB bytes in the swizzled layout the
     // MMA's B operand expects (latent-major rows), the lo half M rows after the hi half.
     {
-        const float *Zg = a.Z + ((size_t)b * a.H + h) * M * DR;
+        const float *Zg = a.Z + (((size_t)b * a.H + h) * a.mtot + a.m0) * DR;
         if (kHalf) {   // upper halves of the rows of Q, Z_hi and Z_lo are zero
             for (int i = threadIdx.x; i < M * (D / 8); i += kTcThreads) {
                 reinterpret_cast<uint4 *>(sQ)[i] = make_uint4(0, 0, 0, 0);
@@ -315,13 +318,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
             __syncthreads();
             if constexpr (DR == 4) {
-                stage_rows4<D>(sQ, a.Q + (size_t)h * M * DR, M, off);
+                stage_rows4<D>(sQ, a.Q + ((size_t)h * a.mtot + a.m0) * DR, M, off);
                 stage_rows4_hilo<D>(sZ, sZ + (size_t)M * G::RB, Zg, M, off);
             } else {
                 for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
                     const int m = i / (DR / 8), c = i % (DR / 8);
                     *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) =
-                        *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + c * 8);
+                        *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * a.mtot + a.m0 + m) * DR + c * 8);
                 }
             }
         }
@@ -358,7 +361,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 // Q_h: M/16 boxes of 16 rows
                 ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
                 for (int r = 0; r < M; r += 16)
-                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * a.mtot + a.m0 + r);
             }
             for (int i = 0; i < ntiles; ++i) {
                 const int s = i % nstages;
@@ -532,7 +535,19 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                 }
-                if (DR == 4) {
+                if (a.Ypart != nullptr) {                       // a range of the latents: float32 rows for the combine kernel
+                    if (n < a.N) {
+                        float4 *pd = reinterpret_cast<float4 *>(a.Ypart + (((size_t)b * a.N + n) * a.H + h) * DR + dc * 16);
+                        if (DR == 4) {
+                            pd[0] = make_float4((off ? y[4] : y[0]) * inv, (off ? y[5] : y[1]) * inv,
+                                                (off ? y[6] : y[2]) * inv, (off ? y[7] : y[3]) * inv);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < (DR < 16 ? DR : 16) / 4; ++k)
+                                pd[k] = make_float4(y[4 * k] * inv, y[4 * k + 1] * inv, y[4 * k + 2] * inv, y[4 * k + 3] * inv);
+                        }
+                    }
+                } else if (DR == 4) {
                     if (n < a.N)
                         *reinterpret_cast<uint2 *>(dst) =
                             make_uint2(ptx::pack_bf16((off ? y[4] : y[0]) * inv, (off ? y[5] : y[1]) * inv),
@@ -560,6 +575,52 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         ptx::tmem_dealloc(tm, (uint32_t)pl.ncols);
     }
     if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
+}
+
+// Decode over more latents than one launch holds: every launch decodes a range of the latents into float32 rows
+// normalised over that range (Ypart[c]) with the range's log-sum-exp (lse_part[c]); this kernel joins the C ranges,
+//   lse = log sum_c exp(lse_c),   Y = sum_c exp(lse_c - lse) Ypart[c],
+// the same algebra as the split-N merge of the encode stage.  One thread per (token, head) row of DR elements.
+template <int DR>
+__global__ void __launch_bounds__(256)
+decode_combine_kernel(const float *__restrict__ Ypart, const float *__restrict__ lse_part, int C, long rows,
+                      __nv_bfloat16 *__restrict__ Y, float *__restrict__ lse_dec) {
+    const long row = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    float lc[4], mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        lc[c] = c < C ? lse_part[(size_t)c * rows + row] : -INFINITY;
+        mx = fmaxf(mx, lc[c]);
+    }
+    float w[4], sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        w[c] = c < C ? expf(lc[c] - mx) : 0.f;
+        sum += w[c];
+    }
+    const float inv = 1.f / sum;
+    float y[DR];
+#pragma unroll
+    for (int k = 0; k < DR; ++k) y[k] = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        if (c < C) {
+            const float4 *src = reinterpret_cast<const float4 *>(Ypart + ((size_t)c * rows + row) * DR);
+#pragma unroll
+            for (int k = 0; k < DR / 4; ++k) {
+                const float4 v = src[k];
+                y[4 * k] = fmaf(w[c], v.x, y[4 * k]);
+                y[4 * k + 1] = fmaf(w[c], v.y, y[4 * k + 1]);
+                y[4 * k + 2] = fmaf(w[c], v.z, y[4 * k + 2]);
+                y[4 * k + 3] = fmaf(w[c], v.w, y[4 * k + 3]);
+            }
+        }
+    }
+    uint32_t *dst = reinterpret_cast<uint32_t *>(Y + (size_t)row * DR);
+#pragma unroll
+    for (int k = 0; k < DR / 2; ++k) dst[k] = ptx::pack_bf16(y[2 * k] * inv, y[2 * k + 1] * inv);
+    if (lse_dec != nullptr) lse_dec[row] = mx + logf(sum);
 }
 
 // ------------------------------------------------------------------------------------------------ encode
