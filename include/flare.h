@@ -125,7 +125,8 @@ int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, co
  * bfloat16 inputs run all three passes (dZ; dK, dV; dQ_lat) on the tensor cores (the last two for D <= 32), with
  * every rounded factor of a cancelling sum carried as two bfloat16 halves; float32 inputs run on the CUDA cores.
  * dQ_lat, dK, dV are overwritten.  Workspace: flare_workspace_bytes(desc, FLARE_OP_BACKWARD) bytes holding dZ,
- * per-split partial sums of dZ and dQ_lat, and one float per (b, n, h); nothing of size N x M.
+ * per-split partial sums of dZ and dQ_lat, one float per (b, n, h), and, beyond 512 bfloat16 latents (256 at
+ * D = 32), float32 sums of the rows of dK and dV; nothing of size N x M.
  */
 int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
                    const uint8_t *key_mask, const void *Y, const void *dY, const float *Z, const float *lse_enc,

@@ -263,10 +263,12 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     return FLARE_OK;
 }
 
-template <int D, int DRT = 0>
+template <int D, int DRT = 0, int kMode = 0>
 int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
                         const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
-                        const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st) {
+                        const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st,
+                        int m0 = 0, int mc = 0, float *kvacc = nullptr) {
+    if (mc == 0) mc = d->M;                                     // the launch's range of latents: [m0, m0 + mc)
     CUtensorMap tmK, tmV, tmG, tmQ;
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
@@ -275,24 +277,25 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     BwdTokTcArgs a;
-    a.stages = BwdTokSmem<D>::stages(d->M);
+    a.stages = BwdTokSmem<D>::stages(mc);
     if (a.stages < 1) return FLARE_ERR_UNSUPPORTED;
-    const size_t smem = BwdTokSmem<D>::total(a.stages, d->M);
+    const size_t smem = BwdTokSmem<D>::total(a.stages, mc);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.dZ = dZ; a.lse_enc = lse_enc; a.de = de; a.lse_dec = lse_dec; a.key_mask = mask;
     a.dK = (__nv_bfloat16 *)dK; a.dV = (__nv_bfloat16 *)dV; a.dd = dd; a.status = status;
-    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = mc;
+    a.mtot = d->M; a.m0 = m0; a.first = m0 == 0; a.last = m0 + mc >= d->M; a.kvacc = kvacc;
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = (d->N + kTile - 1) / kTile;
     long per_head = sms / ((long)d->B * d->H);
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
-    bwd_token_tc_kernel<D, DRT><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_token_tc_kernel<D, DRT, kMode><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -399,9 +402,14 @@ SimtPlan bwd_dq_plan(const flare_desc_t *d, int sms) {
 }
 
 struct BwdLayout {
-    size_t part, dz, de, dd, total;
+    size_t part, dz, de, dd, kvacc, total;
     int P;
 };
+
+// Latents one launch of the tensor-core token kernel keeps in shared memory (five operands of D-wide bf16 rows,
+// beside at least five tile stages); more are worked off in ranges of this many.
+int token_range(const flare_desc_t *d) { return d->D == 32 ? 256 : 512; }
+bool token_in_ranges(const flare_desc_t *d) { return bwd_dq_on_tensor_cores(d) && d->M > token_range(d); }
 
 BwdLayout bwd_layout(const flare_desc_t *d, int sms) {
     BwdLayout w;
@@ -415,6 +423,8 @@ BwdLayout bwd_layout(const flare_desc_t *d, int sms) {
     w.dz = off;   off += align_up(sizeof(float) * (size_t)rows * d->D);
     w.de = off;   off += align_up(sizeof(float) * (size_t)rows);
     w.dd = off;   off += align_up(sizeof(float) * (size_t)d->B * d->N * d->H);
+    w.kvacc = off;                                             // float32 sums of the rows of dK and dV over latent ranges
+    if (token_in_ranges(d)) off += align_up(sizeof(float) * 2 * (size_t)d->B * d->N * d->H * d->D);
     w.total = off;
     return w;
 }
@@ -465,10 +475,26 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     bool tok_on_tc = false;
     if constexpr (std::is_same<T, __nv_bfloat16>::value && D <= 32) {
         constexpr int DK = D < 16 ? 16 : D;                     // width the kernels multiply (D < 16: narrow forms)
-        if (bwd_dq_on_tensor_cores(d) && BwdTokSmem<DK>::stages(d->M) >= 1) {
-            const int rc = launch_bwd_token_tc<DK, (D < 16 ? D : 0)>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd,
-                                                  reinterpret_cast<uint32_t *>(ws), st);
+        constexpr int DRT = D < 16 ? D : 0;
+        uint32_t *status = reinterpret_cast<uint32_t *>(ws);
+        if (bwd_dq_on_tensor_cores(d) && !token_in_ranges(d) && BwdTokSmem<DK>::stages(d->M) >= 1) {
+            const int rc = launch_bwd_token_tc<DK, DRT>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd,
+                                                        status, st);
             if (rc != FLARE_OK) return rc;
+            tok_on_tc = true;
+        } else if (token_in_ranges(d)) {
+            // two series of launches over the latent ranges: dd[n] first, then the rows of dK and dV
+            float *kvacc = reinterpret_cast<float *>(ws + w.kvacc);
+            const int R = token_range(d);
+            for (int mode = 1; mode <= 2; ++mode)
+                for (int m0 = 0; m0 < d->M; m0 += R) {
+                    const int mc = d->M - m0 < R ? d->M - m0 : R;
+                    const int rc = mode == 1 ? launch_bwd_token_tc<DK, DRT, 1>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec,
+                                                                              dK, dV, dd, status, st, m0, mc, kvacc)
+                                             : launch_bwd_token_tc<DK, DRT, 2>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec,
+                                                                              dK, dV, dd, status, st, m0, mc, kvacc);
+                    if (rc != FLARE_OK) return rc;
+                }
             tok_on_tc = true;
         }
     }

@@ -390,9 +390,16 @@ struct BwdTokTcArgs {
     const float *lse_dec;      // [B,N,H]
     const uint8_t *key_mask;   // [B,N] or null
     __nv_bfloat16 *dK, *dV;    // [B,N,H,D]
-    float *dd;                 // [B,H,N] out (workspace)
+    float *dd;                 // [B,H,N] (workspace): written in modes 0 and 1, read in mode 2
     uint32_t *status;
-    int B, H, N, M;
+    int B, H, N, M;            // M: latents this launch works on (all of them, or a range)
+    int mtot, m0;              // latents per head in memory, and the first one of this launch's range
+    // More latents than one launch can keep in shared memory are worked off in ranges, by two series of launches:
+    // mode 1 (first sweep only) adds the range's share of dd[n] to the workspace; mode 2 (second sweep only, dd
+    // complete) adds the range's share of the rows of dK and dV to float32 sums in kvacc [2][B*N*H][D] and, in the
+    // last range, writes the rows.  Mode 0 does both sweeps over all latents in one launch.
+    int first, last;           // (the mode is a template parameter of the kernel)
+    float *kvacc;
     float scale, sl2;
     int tiles, stages;
 };
@@ -422,7 +429,7 @@ struct BwdTokSmem {
 // grid = (CTAs per head, H, B); a CTA takes the token tiles blockIdx.x, blockIdx.x + gridDim.x, ...
 // DRT = 8 or 4 (with D = 16): the narrow form (head DRT wide in memory; only the head's columns of the rows of dK
 // and dV are kept).
-template <int D, int DRT = 0>
+template <int D, int DRT = 0, int kMode = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdTokTcArgs a) {
@@ -473,22 +480,22 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (kHalf) {
         __syncthreads();
         if constexpr (DR == 4) {
-            const size_t r0 = ((size_t)b * a.H + h) * M;
-            stage_rows4<D>(sQ, a.Q + (size_t)h * M * DR, M, off);
+            const size_t r0 = ((size_t)b * a.H + h) * a.mtot + a.m0;
+            stage_rows4<D>(sQ, a.Q + ((size_t)h * a.mtot + a.m0) * DR, M, off);
             stage_rows4_hilo<D>(smem + SM::lat_off(stages, M, 1), smem + SM::lat_off(stages, M, 2), a.Z + r0 * DR, M, off);
             stage_rows4_hilo<D>(smem + SM::lat_off(stages, M, 3), smem + SM::lat_off(stages, M, 4), a.dZ + r0 * DR, M, off);
         } else {
             for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
                 const int m = i / (DR / 8), ch = i % (DR / 8);
                 *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
-                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + m) * DR + ch * 8);
+                    *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * a.mtot + a.m0 + m) * DR + ch * 8);
             }
         }
     }
     for (int m = threadIdx.x; m < MU; m += kTcThreads) {
         float nle = -INFINITY, nde = 0.f;
         if (m < M) {
-            const size_t r = ((size_t)b * a.H + h) * M + m;
+            const size_t r = ((size_t)b * a.H + h) * a.mtot + a.m0 + m;
             const float le = a.lse_enc[r];
             nle = (le == -INFINITY) ? -INFINITY : -le * 1.4426950408889634f;
             nde = -a.de[r];
@@ -499,7 +506,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     constexpr int ZC = DR >= 8 ? DR / 8 : 1;                    // 8-float chunks per row (none for DR = 4: staged above)
     for (int i = threadIdx.x; i < (DR >= 8 ? 2 * M * ZC : 0); i += kTcThreads) {
         const int which = i / (M * ZC), rem = i % (M * ZC), m = rem / ZC, ch = rem % ZC;
-        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * M + m) * DR + ch * 8;
+        const float *src = (which == 0 ? a.Z : a.dZ) + (((size_t)b * a.H + h) * a.mtot + a.m0 + m) * DR + ch * 8;
         const float4 lo4 = *reinterpret_cast<const float4 *>(src), hi4 = *reinterpret_cast<const float4 *>(src + 4);
         const float z[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
         uint32_t vh[4], vl[4];
@@ -525,7 +532,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             } else {
                 ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
                 for (int r = 0; r < M; r += 16)
-                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + r);
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * a.mtot + a.m0 + r);
             }
             for (int i = 0; i < nt; ++i) {
                 const int s = i % stages, t = blockIdx.x + i * gridDim.x;
@@ -556,7 +563,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const uint64_t kdesc = ptx::smem_desc(tbase, 16, G::SBO, G::SWZ);
                 const uint64_t vdesc = ptx::smem_desc(tbase + G::TILE_BYTES, 16, G::SBO, G::SWZ);
                 const uint64_t gdesc = ptx::smem_desc(tbase + 2 * G::TILE_BYTES, 16, G::SBO, G::SWZ);
-                for (int sweep = 0; ok && sweep < 2; ++sweep) {
+                for (int sweep = (kMode == 2 ? 1 : 0); ok && sweep < (kMode == 1 ? 1 : 2); ++sweep) {
                     for (int u = 0; u < nu; ++u) {
                         const uint64_t uoff = (uint64_t)(u * UNIT * G::RB / 16);      // the unit's latent rows
                         uint64_t ld[5];
@@ -602,7 +609,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 }
                 if (!ok) break;
                 ptx::mma_commit(bar(T_EMPTY + s));
-                ptx::mma_commit(bar(ACC_FULL + g));
+                if (kMode != 1) ptx::mma_commit(bar(ACC_FULL + g));
             }
         }
     } else {
@@ -634,37 +641,61 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             ptx::tc_fence_before();
             ptx::mbar_arrive(bar(ACC_FREE + g));
             if (p_inside) {
-                a.dd[p_ddi] = p_dd;
-                uint4 *dk = reinterpret_cast<uint4 *>(a.dK + p_tok * DR), *dv = reinterpret_cast<uint4 *>(a.dV + p_tok * DR);
-                if (DR == 4) {
-                    auto k4 = [&](int i) { return __uint_as_float(off ? ak[4 + i] : ak[i]) * a.scale; };
-                    auto v4 = [&](int i) { return __uint_as_float(off ? avv[4 + i] : avv[i]); };
-                    *reinterpret_cast<uint2 *>(dk) = make_uint2(ptx::pack_bf16(k4(0), k4(1)), ptx::pack_bf16(k4(2), k4(3)));
-                    *reinterpret_cast<uint2 *>(dv) = make_uint2(ptx::pack_bf16(v4(0), v4(1)), ptx::pack_bf16(v4(2), v4(3)));
+                if (kMode == 0) a.dd[p_ddi] = p_dd;
+                float fk[DR], fv[DR];
+#pragma unroll
+                for (int i = 0; i < DR; ++i) {                  // the head's columns of the accumulators
+                    fk[i] = __uint_as_float((DR == 4 && off) ? ak[(4 + i) % D] : ak[i]);
+                    fv[i] = __uint_as_float((DR == 4 && off) ? avv[(4 + i) % D] : avv[i]);
                 }
+                float4 *sk = reinterpret_cast<float4 *>(a.kvacc + p_tok * DR);
+                float4 *sv = reinterpret_cast<float4 *>(a.kvacc + ((size_t)a.B * a.N * a.H + p_tok) * DR);
+                if (kMode == 2 && !a.first) {                  // the earlier ranges' shares
 #pragma unroll
-                for (int q = 0; q < DR / 8; ++q) {
-                    uint32_t wk[4], wv4[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        wk[k] = ptx::pack_bf16(__uint_as_float(ak[8 * q + 2 * k]) * a.scale, __uint_as_float(ak[8 * q + 2 * k + 1]) * a.scale);
-                        wv4[k] = ptx::pack_bf16(__uint_as_float(avv[8 * q + 2 * k]), __uint_as_float(avv[8 * q + 2 * k + 1]));
+                    for (int i = 0; i < DR / 4; ++i) {
+                        const float4 pk4 = sk[i], pv4 = sv[i];
+                        fk[4 * i] += pk4.x; fk[4 * i + 1] += pk4.y; fk[4 * i + 2] += pk4.z; fk[4 * i + 3] += pk4.w;
+                        fv[4 * i] += pv4.x; fv[4 * i + 1] += pv4.y; fv[4 * i + 2] += pv4.z; fv[4 * i + 3] += pv4.w;
                     }
-                    dk[q] = make_uint4(wk[0], wk[1], wk[2], wk[3]);
-                    dv[q] = make_uint4(wv4[0], wv4[1], wv4[2], wv4[3]);
+                }
+                if (kMode == 2 && !a.last) {
+#pragma unroll
+                    for (int i = 0; i < DR / 4; ++i) {
+                        sk[i] = make_float4(fk[4 * i], fk[4 * i + 1], fk[4 * i + 2], fk[4 * i + 3]);
+                        sv[i] = make_float4(fv[4 * i], fv[4 * i + 1], fv[4 * i + 2], fv[4 * i + 3]);
+                    }
+                } else {
+                    uint32_t *dk = reinterpret_cast<uint32_t *>(a.dK + p_tok * DR), *dv = reinterpret_cast<uint32_t *>(a.dV + p_tok * DR);
+                    uint32_t wk[DR / 2], wv[DR / 2];
+#pragma unroll
+                    for (int i = 0; i < DR / 2; ++i) {
+                        wk[i] = ptx::pack_bf16(fk[2 * i] * a.scale, fk[2 * i + 1] * a.scale);
+                        wv[i] = ptx::pack_bf16(fv[2 * i], fv[2 * i + 1]);
+                    }
+                    if (DR == 4) {
+                        *reinterpret_cast<uint2 *>(dk) = make_uint2(wk[0], wk[1]);
+                        *reinterpret_cast<uint2 *>(dv) = make_uint2(wv[0], wv[1]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < DR / 8; ++q) {
+                            reinterpret_cast<uint4 *>(dk)[q] = make_uint4(wk[4 * q], wk[4 * q + 1], wk[4 * q + 2], wk[4 * q + 3]);
+                            reinterpret_cast<uint4 *>(dv)[q] = make_uint4(wv[4 * q], wv[4 * q + 1], wv[4 * q + 2], wv[4 * q + 3]);
+                        }
+                    }
                 }
             }
             pend = false;
             return true;
         };
         // this lane's token of a tile: its decode log-sum-exp and mask byte, fetched one tile ahead
-        float f_ld = 0.f;
+        float f_ld = 0.f, f_dd = 0.f;
         uint32_t f_mask = 1u;
         auto fetch = [&](int i) {
             const int n = (blockIdx.x + i * gridDim.x) * kTile + row;
             const size_t nn = (size_t)b * a.N + (n < a.N ? n : 0);
             f_ld = a.lse_dec[nn * a.H + h];
             f_mask = a.key_mask == nullptr ? 1u : (uint32_t)a.key_mask[nn];
+            if (kMode == 2) f_dd = a.dd[((size_t)b * a.H + h) * a.N + (n < a.N ? n : 0)];
         };
         if (g < ng && g < nt) fetch(g);
         for (int i = g; ok && g < ng && i < nt; i += ng, ++k_tile) {
@@ -674,11 +705,12 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const size_t tok = ((size_t)b * a.N + (inside ? n : 0)) * a.H + h;
             const float negld = inside ? -f_ld * 1.4426950408889634f : -INFINITY;
             const float2 negldp = make_float2(negld, negld);
+            const float dd_given = inside ? f_dd : 0.f;         // mode 2: dd[n] over all latents, from the workspace
             if (i + ng < nt) fetch(i + ng);
             const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;      // uniform over the group
             // sweep 1: dd[n] = sum_m W_dec[n,m] (dY_n . Z_m)
             float2 dd2 = make_float2(0.f, 0.f);
-            for (int u = 0; ok && u < nu; ++u) {
+            for (int u = 0; ok && kMode != 2 && u < nu; ++u) {
                 if (!warp_wait(bar(S_FULL + g), cnt & 1, abort_flag, kErrBwdTok | 6)) { ok = false; break; }
                 ++cnt;
                 ptx::tc_fence_after();
@@ -698,8 +730,15 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(bar(P_FULL + g));
             }
-            const float dd = dd2.x + dd2.y;
+            const float dd = kMode == 2 ? dd_given : dd2.x + dd2.y;
             const float2 negddp = make_float2(-dd, -dd);
+            if (kMode == 1) {                                  // this range's share of dd[n]; no second sweep
+                if (inside) {
+                    const size_t ddi = ((size_t)b * a.H + h) * a.N + n;
+                    a.dd[ddi] = (a.first ? 0.f : a.dd[ddi]) + dd;
+                }
+                continue;
+            }
             if (ok && pend) ok = write_rows();                  // the previous tile's rows
             // sweep 2: dS^T and W_enc^T of every unit, handed to the issuing warp
             auto unit2 = [&](auto masked, int u) {
