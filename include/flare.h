@@ -90,7 +90,10 @@ int flare_encode_partials(const flare_desc_t *desc);
 
 /*
  * Encode (Section 3.2, encode equation; per-latent sum of the design-principles appendix):
- * Z and, if lse_enc != NULL, lse_enc.  Split over N: every CTA keeps a running maximum and sum per latent
+ * Z and, if lse_enc != NULL, lse_enc.  Asking for lse_enc marks a forward whose Z will be differentiated through:
+ * for bfloat16 inputs the softmax weights then enter the value contraction as two bfloat16 halves (Z within about
+ * 1e-4 of its RMS instead of 4e-3, a quarter more time in this stage), because the backward magnifies the error
+ * of Z several times.  Split over N: every CTA keeps a running maximum and sum per latent
  * (online softmax) over its token range; a second kernel merges the splits by log-sum-exp.
  */
 int flare_encode(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,

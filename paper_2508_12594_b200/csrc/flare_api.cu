@@ -203,7 +203,7 @@ int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
 constexpr float kLog2e = 1.4426950408889634f;
 
 // kDz: the backward's dZ form of the kernel (V is then dY, lse_dec the decode log-sum-exp rows, pm and pl unused).
-template <int D, bool kPair, bool kDz = false, int DRT = 0>
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false>
 int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
                      const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
                      const float *lse_dec = nullptr) {
@@ -217,7 +217,7 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     const size_t smem = EncodeSmem<DG>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     EncodeTcArgs a;
@@ -228,7 +228,7 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair, kDz, DRT><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -573,15 +573,19 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
     if (use_tc(d)) {
         TcEncodePlan p = tc_encode_plan(d, di.sms);
         uint32_t *status = reinterpret_cast<uint32_t *>(base);
+        // a caller that asks for lse_enc is saving Z for the backward: weights as two bf16 halves (see exp_chunk_hilo)
+#define FLARE_ENC(DD, PAIR, DRT)                                                                                         \
+    (lse_enc != nullptr ? launch_encode_tc<DD, PAIR, false, DRT, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st) \
+                        : launch_encode_tc<DD, PAIR, false, DRT, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st))
         if (encode_head_pairs(d))
-            rc = d->D == 16 ? launch_encode_tc<16, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-                            : launch_encode_tc<32, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
+            rc = d->D == 16 ? FLARE_ENC(16, true, 0) : FLARE_ENC(32, true, 0);
         else
-            rc = d->D == 4    ? launch_encode_tc<16, false, false, 4>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-                 : d->D == 8  ? launch_encode_tc<16, false, false, 8>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-                 : d->D == 16 ? launch_encode_tc<16, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-                 : d->D == 32 ? launch_encode_tc<32, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st)
-                              : launch_encode_tc<64, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
+            rc = d->D == 4    ? FLARE_ENC(16, false, 4)
+                 : d->D == 8  ? FLARE_ENC(16, false, 8)
+                 : d->D == 16 ? FLARE_ENC(16, false, 0)
+                 : d->D == 32 ? FLARE_ENC(32, false, 0)
+                              : FLARE_ENC(64, false, 0);
+#undef FLARE_ENC
     } else {
         SimtPlan p = simt_plan(d, di.sms);
         rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)

@@ -137,6 +137,28 @@ __device__ __forceinline__ void exp_chunk(const uint32_t *r, uint32_t *pk, float
     }
 }
 
+// exp_chunk with the weights leaving as two bf16 halves (hi = round(p), lo = round(p - hi)), for an encode whose Z
+// is saved for the backward: the gradients magnify the error of Z several times, and with single bf16 weights
+// (Z off by 3e-3 to 4e-3 of its RMS) that alone put dK and dQ at 2e-2 to 3e-2 of theirs where N is only a few
+// times M (measured; with the exact Z the same backward is at 5e-4).
+template <int NV, bool kMasked>
+__device__ __forceinline__ void exp_chunk_hilo(const uint32_t *r, uint32_t *hi, uint32_t *lo, float2 sl2p, float2 negp,
+                                               float2 &sum2, uint32_t valid = 0xffffffffu, bool dead = false) {
+#pragma unroll
+    for (int k = 0; k < NV / 2; ++k) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * k]), __uint_as_float(r[2 * k + 1])), sl2p, negp);
+        float2 p = make_float2(ptx::ex2(x.x), ptx::ex2(x.y));
+        if (kMasked) {
+            if (dead || !((valid >> (2 * k)) & 1)) p.x = 0.f;
+            if (dead || !((valid >> (2 * k + 1)) & 1)) p.y = 0.f;
+        }
+        sum2 = __fadd2_rn(sum2, p);
+        const uint32_t h = ptx::pack_bf16(p.x, p.y);
+        hi[k] = h;
+        lo[k] = ptx::pack_bf16(p.x - __uint_as_float(h << 16), p.y - __uint_as_float(h & 0xffff0000u));
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ decode
 // How the four softmax groups share tensor memory in decode.  `cs` groups split the M score columns of one
 // buffer into ranges of `part_w` columns (the last may be shorter); `nbuf` buffers of `cb` columns hold
@@ -677,7 +699,9 @@ struct EncodeSmem {
 // Narrow form (DRT = 8 or 4 with D = 16; not with kPair): the head is DRT wide in memory, as in the decode kernel:
 // K and V tile rows carry the neighbouring heads' features beside the head's own, Q rows zeros there; accumulator
 // columns outside the head's (weights times the neighbours' values) are dropped.
-template <int D, bool kPair, bool kDz = false, int DRT = 0>
+//
+// kHiLo: the weights go to the value contraction as two bf16 halves (see exp_chunk_hilo), as in the dZ form.
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
@@ -828,7 +852,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int k = 0; k < UNIT / 16; ++k) {
                     ptx::mma_ts(dcol, gcol + w * UNIT + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, (n > 0 || k > 0) ? 1u : 0u);
-                    if (kDz)    // the lo halves of the weights sit 16 columns further on
+                    if (kDz || kHiLo)    // the lo halves of the weights sit 16 columns further on
                         ptx::mma_ts(dcol, gcol + w * UNIT + 16 + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, 1u);
                 }
                 ptx::mma_commit(bar(PV_DONE + g));
@@ -922,8 +946,15 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const float neg = dead ? 0.f : -m_run * a.sl2;
             const float2 negp = make_float2(neg, neg);
             uint32_t pk[16];
-            exp_chunk<32, kMasked>(r, pk, sl2p, negp, l2, wv, dead);
-            ptx::tmem_st16(sbase, pk);
+            if (kHiLo) {
+                uint32_t pl[16];
+                exp_chunk_hilo<32, kMasked>(r, pk, pl, sl2p, negp, l2, wv, dead);
+                ptx::tmem_st16(sbase, pk);                      // hi halves over the first 16 score columns,
+                ptx::tmem_st16(sbase + 16, pl);                 // lo halves over the other 16
+            } else {
+                exp_chunk<32, kMasked>(r, pk, sl2p, negp, l2, wv, dead);
+                ptx::tmem_st16(sbase, pk);
+            }
             ptx::tmem_wait_st();                                // weights (and a rescaled accumulator) are in place
             ptx::tc_fence_before();
             ptx::mbar_arrive(bar(P_FULL + 2 * g + w));

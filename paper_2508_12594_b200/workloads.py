@@ -55,6 +55,9 @@ CONFIGS = {
     "padded": Workload("padded", B=32, H=4, N=4096, M=128, D=32, dtype="bf16", kind="padded", seed=3,
                        backward=True),
     "mesh3d_1m": Workload("mesh3d_1m", B=1, H=8, N=1048576, M=256, D=16, dtype="bf16", kind="cube", seed=4),
+    # the shape of the paper's own million-point study (field-prediction appendix): C = 64, H = 8, hence D = 8,
+    # with M between 128 and 2048 latents; not one of the five benchmark workloads
+    "field_1m": Workload("field_1m", B=1, H=8, N=1048576, M=1024, D=8, dtype="bf16", kind="cube", seed=6, backward=True),
 }
 
 SWEEP_N = (16384, 131072, 1048576)

@@ -136,12 +136,19 @@ def test_encode_then_decode_equals_forward(oracle):
     flare.flare_decode(desc, Q, K, Zo, Y2, None)
     torch.cuda.synchronize()
     assert rel_err(to_np64(Y2), ref["Y"]) <= TOL["bf16"]
-    # optional outputs may be NULL; Z may live in the workspace
+    # optional outputs may be NULL; Z may live in the workspace.  Without lse_enc the encode weights are single
+    # bfloat16 values (with it, two halves, for a Z fit to be differentiated through), so Y agrees with the
+    # oracle to the same bound but not bit for bit with Y1.
     wsf = flare.alloc_workspace(desc, flare.OP_FORWARD)
     Y3 = torch.empty_like(Y1)
     flare.flare_forward(desc, Q, K, V, mask, Y3, None, None, None, wsf)
     torch.cuda.synchronize()
-    assert torch.equal(Y1, Y3)
+    assert rel_err(to_np64(Y3), ref["Y"]) <= TOL["bf16"]
+    assert rel_err(to_np64(Y3), to_np64(Y1)) <= TOL["bf16"]
+    Y4 = torch.empty_like(Y1)
+    flare.flare_forward(desc, Q, K, V, mask, Y4, None, None, None, wsf)
+    torch.cuda.synchronize()
+    assert torch.equal(Y3, Y4)
 
 
 def test_error_paths_on_device():

@@ -24,6 +24,9 @@ FULL = [
     workloads.sweep_point(131072, 32),
     workloads.sweep_point(131072, 128),
     workloads.sweep_point(131072, 512),
+    # the paper's million-point shape (head width 8, 1024 latents: narrow kernels, decode in latent ranges), cut to
+    # a length the oracle encodes in seconds
+    workloads.CONFIGS["field_1m"].with_(N=65536, name="field_1m@N=65536"),
 ]
 
 
@@ -51,7 +54,8 @@ def test_forward_full_size_sampled(oracle, w):
 
 
 BACKWARD_FULL = [workloads.CONFIGS["padded"], workloads.CONFIGS["mesh2d"].with_(backward=True),
-                 workloads.sweep_point(131072, 128)]
+                 workloads.sweep_point(131072, 128),
+                 workloads.CONFIGS["field_1m"].with_(N=8192, name="field_1m@N=8192")]
 
 
 @pytest.mark.parametrize("w", BACKWARD_FULL, ids=lambda w: w.name)
