@@ -300,7 +300,7 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     return FLARE_OK;
 }
 
-template <int D, int DRT = 0>
+template <int D, int DRT = 0, bool kPart = false>
 int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
                      float *lse_dec, uint32_t *status, cudaStream_t st, int m0 = 0, int mc = 0, float *Ypart = nullptr) {
     if (mc == 0) mc = d->M;                                     // the launch's range of latents: [m0, m0 + mc)
@@ -312,7 +312,7 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     const size_t smem = DecodeSmem<D>::total(mc);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT, kPart>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     DecodeTcArgs a;
@@ -328,7 +328,7 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
     dim3 grid((unsigned)per_head, d->H, d->B);
-    decode_tc_kernel<D, DRT><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
+    decode_tc_kernel<D, DRT, kPart><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -625,7 +625,7 @@ int decode_tc_any(const flare_desc_t *d, int sms, const void *Q, const void *K, 
     float *lpart = reinterpret_cast<float *>(range_scratch + align_up(sizeof(float) * C * rows * d->D));
     for (int c = 0; c < C; ++c) {
         const int m0 = c * kDecodeMaxM, mc = d->M - m0 < kDecodeMaxM ? d->M - m0 : kDecodeMaxM;
-        const int rc = launch_decode_tc<D, DRT>(d, sms, Q, K, Z, nullptr, lpart + (size_t)c * rows, status, st, m0, mc,
+        const int rc = launch_decode_tc<D, DRT, true>(d, sms, Q, K, Z, nullptr, lpart + (size_t)c * rows, status, st, m0, mc,
                                                 Ypart + (size_t)c * rows * DR);
         if (rc != FLARE_OK) return rc;
     }

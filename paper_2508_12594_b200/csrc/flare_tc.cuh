@@ -236,8 +236,8 @@ struct DecodeTcArgs {
     uint32_t *status;    // workspace header or null
     int B, H, N, M;      // M: latents this launch works on (all of them, or a range of at most 512)
     int mtot, m0;        // latents per head in Q and Z, and the first one of this launch's range
-    float *Ypart;        // null, or [B,N,H,D] float32: rows normalised over the range go here instead of Y, with
-                         // their log-sum-exp in lse_dec, for decode_combine_kernel
+    float *Ypart;        // kPart form of the kernel: [B,N,H,D] float32, rows normalised over the range go here instead
+                         // of Y, with their log-sum-exp in lse_dec, for decode_combine_kernel
     float sl2;           // scale * log2(e)
     int tiles;           // ceil(N / 128)
     DecodePlan plan;
@@ -272,7 +272,7 @@ struct DecodeSmem {
 //
 // Narrow form (DRT = 8 or 4 with D = 16): the head is DRT wide in memory (see narrow_offset).  This is how head
 // widths below the smallest MMA K-step (16) run on the tensor cores.
-template <int D, int DRT = 0>
+template <int D, int DRT = 0, bool kPart = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
     constexpr bool kHalf = DRT != 0;
@@ -557,7 +557,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                 }
-                if (a.Ypart != nullptr) {                       // a range of the latents: float32 rows for the combine kernel
+                if (kPart) {                                    // a range of the latents: float32 rows for the combine kernel
                     if (n < a.N) {
                         float4 *pd = reinterpret_cast<float4 *>(a.Ypart + (((size_t)b * a.N + n) * a.H + h) * DR + dc * 16);
                         if (DR == 4) {
