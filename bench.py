@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised under profiles/ (taken on a 262,144-token slice and scaled by 4: traffic is proportional to N).
 # Valid for the kernels as profiled; set to None when a kernel changes until the capture is redone.
 NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.321152e6 + 3.520256e6),
-               ("mesh3d_1m", "decode"): 4 * (67.415296e6 + 29.168128e6)}
+               ("mesh3d_1m", "decode"): 4 * (67.362816e6 + 29.085184e6)}
 
 
 def get_workload(name: str) -> workloads.Workload:
