@@ -80,8 +80,8 @@ const char *flare_last_cuda_error(void);
  * Bytes of scratch `workspace` the given operation needs for `desc` on the current device (0 for an invalid
  * or unsupported descriptor).  Encode writes per-split partial results (running maximum, sum and
  * un-normalised latent rows) there: O(splits * B * H * M * (D + 2)) floats, never anything of size N x M.
- * The forward over more than 512 bfloat16 latents decodes them in ranges of 512 and adds one float32 row and
- * one log-sum-exp per token, head and range: ceil(M / 512) * B * N * H * (D + 1) floats.
+ * The forward over more than 512 bfloat16 latents decodes them in ranges of 256 and adds one float32 row and
+ * one log-sum-exp per token, head and range: ceil(M / 256) * B * N * H * (D + 1) floats.
  */
 size_t flare_workspace_bytes(const flare_desc_t *desc, int op);
 

@@ -606,7 +606,8 @@ constexpr int kDecodeMaxM = 512;
 
 // Ranges of latents a decode over more than kDecodeMaxM latents is cut into, and the scratch their partial results
 // take after the encode layout of the forward workspace: float32 rows [C][B*N*H][D] and log-sum-exps [C][B*N*H].
-int decode_ranges(const flare_desc_t *d) { return (d->M + kDecodeMaxM - 1) / kDecodeMaxM; }
+constexpr int kDecodeRange = 256;   // latents per launch when a decode is cut into ranges
+int decode_ranges(const flare_desc_t *d) { return (d->M + kDecodeRange - 1) / kDecodeRange; }
 bool decode_in_ranges(const flare_desc_t *d) { return use_tc(d) && d->M > kDecodeMaxM; }
 size_t decode_range_bytes(const flare_desc_t *d) {
     if (!decode_in_ranges(d)) return 0;
@@ -624,7 +625,7 @@ int decode_tc_any(const flare_desc_t *d, int sms, const void *Q, const void *K, 
     float *Ypart = reinterpret_cast<float *>(range_scratch);
     float *lpart = reinterpret_cast<float *>(range_scratch + align_up(sizeof(float) * C * rows * d->D));
     for (int c = 0; c < C; ++c) {
-        const int m0 = c * kDecodeMaxM, mc = d->M - m0 < kDecodeMaxM ? d->M - m0 : kDecodeMaxM;
+        const int m0 = c * kDecodeRange, mc = d->M - m0 < kDecodeRange ? d->M - m0 : kDecodeRange;
         const int rc = launch_decode_tc<D, DRT, true>(d, sms, Q, K, Z, nullptr, lpart + (size_t)c * rows, status, st, m0, mc,
                                                 Ypart + (size_t)c * rows * DR);
         if (rc != FLARE_OK) return rc;

@@ -609,15 +609,15 @@ decode_combine_kernel(const float *__restrict__ Ypart, const float *__restrict__
                       __nv_bfloat16 *__restrict__ Y, float *__restrict__ lse_dec) {
     const long row = (long)blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= rows) return;
-    float lc[4], mx = -INFINITY;
+    float lc[8], mx = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 8; ++c) {
         lc[c] = c < C ? lse_part[(size_t)c * rows + row] : -INFINITY;
         mx = fmaxf(mx, lc[c]);
     }
-    float w[4], sum = 0.f;
+    float w[8], sum = 0.f;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 8; ++c) {
         w[c] = c < C ? expf(lc[c] - mx) : 0.f;
         sum += w[c];
     }
@@ -626,7 +626,7 @@ decode_combine_kernel(const float *__restrict__ Ypart, const float *__restrict__
 #pragma unroll
     for (int k = 0; k < DR; ++k) y[k] = 0.f;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 8; ++c) {
         if (c < C) {
             const float4 *src = reinterpret_cast<const float4 *>(Ypart + ((size_t)c * rows + row) * DR);
 #pragma unroll
