@@ -92,6 +92,8 @@ EDGE = [
     # more than 512 latents, and far more latents than tokens (a latent row then follows a single token, and the
     # backward's dZ_m . (V_n - Z_m) magnifies whatever error the forward left in Z)
     (1, 2, 200, 2048, 8, "bf16", 0.1),
+    (2, 1, 400, 640, 32, "bf16", 0.0),      # latent ranges 256 + 256 + 128 in the token kernel
+    (1, 2, 300, 1040, 16, "bf16", 0.2),     # 512 + 512 + 16
     (1, 2, 300, 1024, 16, "bf16", 0.0),
     (1, 2, 1000, 2048, 8, "bf16", 0.1),
     # head width 4

@@ -64,6 +64,7 @@ EDGE = [
     (1, 2, 700, 1024, 16, "bf16", 0.0),
     (1, 2, 300, 2048, 8, "bf16", 0.1),
     (2, 1, 400, 640, 32, "bf16", 0.0),
+    (1, 2, 300, 1040, 16, "bf16", 0.2),     # decode ranges 4 x 256 + 16
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 2049, 300, 64, "f32", 0.0),
     (1, 4, 64, 1, 16, "f32", 0.0),
