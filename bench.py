@@ -115,6 +115,24 @@ def oracle_sample(w: workloads.Workload, inp, sample_tokens: int):
     return w.B * n / dt, dt, n, flare_oracle.max_threads()
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time (every multi-GPU number is the maximum over ranks); `dist` is None on one rank."""
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_workload(w, rank: int):
+    """Replicas: every rank draws its own batch from the same recipe (weak scaling), seed offset by the rank."""
+    return w.with_(seed=w.seed + 1000 * rank)
+
+
+def whole_job_value(w, world: int, ms_step: float) -> float:
+    """Tokens per second over all replicas: every rank processes w.tokens per step."""
+    return world * w.tokens / (ms_step / 1e3)
+
+
 def run_reference(args, w):
     """The reference arm: the oracle on the host cores, each step a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -180,7 +198,7 @@ def main():
         torch.cuda.synchronize()
 
     # every rank draws its own batch (weak scaling): same recipe, rank-dependent seed
-    wr = w.with_(seed=w.seed + 1000 * rank)
+    wr = rank_workload(w, rank)
     inp = workloads.make_inputs(wr)
     Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
     mask = None if inp.key_mask is None else inp.key_mask.cuda()
@@ -275,11 +293,8 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     flare.flare_check(ws)
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    value = world * w.tokens / (ms_step / 1e3)
+    ms_step = max_over_ranks(ms_total, dist, "cuda") / args.steps
+    value = whole_job_value(w, world, ms_step)
 
     e2e = None
     if not args.no_e2e:
@@ -308,10 +323,7 @@ def run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V
         flare.flare_forward_host(desc, hQ, hK, hV, hmask, hY, dQ, dK, dV, dmask, dY, ws, stream)
     ev[1].record(stream)
     barrier()
-    t = torch.tensor([ev[0].elapsed_time(ev[1])], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / args.e2e_steps
+    e2e_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), dist, "cuda") / args.e2e_steps
     h2d = 2 * tensor_bytes + w.H * w.M * w.D * e + (0 if mask is None else w.B * w.N)
     return {"value": world * w.tokens / (e2e_ms / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": tensor_bytes, "ms_per_step": e2e_ms}
