@@ -160,3 +160,15 @@ def test_backward_error_paths():
                                      dV.data_ptr(), ws.data_ptr(), ws.numel(), None)
     assert rc == flare.ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("case", [(1, 2, 700, 128, 16, 3.0), (1, 2, 700, 256, 32, 3.0), (1, 4, 600, 64, 8, 4.0),
+                                  (1, 2, 700, 128, 16, 8.0)], ids=lambda c: "B{}H{}N{}M{}D{}k{}".format(*c))
+def test_backward_large_scores(oracle, case):
+    """Scores up to +-170 at scale 1 (keys of standard deviation 3 to 8): every weight is exp(score - log-sum-exp)
+    with the subtraction done before the exponential, so nothing overflows and nothing loses its leading digits."""
+    B, H, N, M, D, k_std = case
+    inp = workloads.make_random(B, H, N, M, D, dtype="bf16", seed=7, with_dy=True, k_std=k_std)
+    got = gpu_backward(inp)
+    assert all(np.isfinite(v).all() for v in got.values())
+    assert_grads_close(got, oracle_backward(oracle, inp), "bf16", str(case))

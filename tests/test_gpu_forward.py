@@ -172,3 +172,12 @@ def test_error_paths_on_device():
                            ws.data_ptr(), ws.numel(), st)
     assert rc == flare.ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("k_std", [3.0, 8.0])
+def test_large_scores(oracle, k_std):
+    """Scores up to +-170 at scale 1: the running maximum is subtracted before every exponential."""
+    inp = workloads.make_random(1, 2, 700, 128, 16, dtype="bf16", seed=7, k_std=k_std)
+    got = gpu_forward(inp, canary=True)
+    assert np.isfinite(got["Y"]).all() and np.isfinite(got["Z"]).all()
+    assert_forward_close(got, oracle_forward(oracle, inp), "bf16", f"k_std={k_std}")
