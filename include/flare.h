@@ -27,7 +27,7 @@
  * by the caller, 16-byte aligned; the library never allocates, frees or keeps them.  Calls enqueue work on
  * `stream` and return without synchronising; outputs are overwritten, never accumulated into.  Two calls may
  * run concurrently on different streams only with different workspaces.  Results are bitwise reproducible
- * for a fixed descriptor on a fixed device.
+ * for a fixed descriptor and set of requested outputs on a fixed device.
  *
  * Supported shapes: D in {4, 8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 2048.
  * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation (D = 8 and 4 as part of a 16-wide
@@ -92,7 +92,7 @@ int flare_encode_partials(const flare_desc_t *desc);
  * Encode (Section 3.2, encode equation; per-latent sum of the design-principles appendix):
  * Z and, if lse_enc != NULL, lse_enc.  Asking for lse_enc marks a forward whose Z will be differentiated through:
  * for bfloat16 inputs the softmax weights then enter the value contraction as two bfloat16 halves (Z within about
- * 1e-4 of its RMS instead of 4e-3, a quarter more time in this stage), because the backward magnifies the error
+ * 1e-4 of its RMS instead of 4e-3, about a sixth more time in this stage), because the backward magnifies the error
  * of Z several times.  Split over N: every CTA keeps a running maximum and sum per latent
  * (online softmax) over its token range; a second kernel merges the splits by log-sum-exp.
  */
