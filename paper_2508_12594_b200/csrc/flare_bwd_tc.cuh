@@ -600,9 +600,9 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                                 const uint32_t acc = (u > 0 || k > 0) ? 1u : 0u;
                                 ptx::mma_ts(kcol, gcol + k * 8, qmn + (uint64_t)(k * G::RB), idescO, acc);              // dS hi
                                 ptx::mma_ts(kcol, gcol + UNIT + k * 8, qmn + (uint64_t)(k * G::RB), idescO, 1u);        // dS lo
-                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 8, zmn + (uint64_t)(k * G::RB), idescO, acc);   // W_enc dZ_hi
-                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 8, zln + (uint64_t)(k * G::RB), idescO, 1u);    // W_enc dZ_lo
-                                ptx::mma_ts(vcol, gcol + UNIT / 2 + k * 8, zmn + (uint64_t)(k * G::RB), idescO, 1u);    // W_enc lo x dZ_hi
+                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 16, zmn + (uint64_t)(k * G::RB), idescO, acc);       // W_enc dZ_hi
+                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 16, zln + (uint64_t)(k * G::RB), idescO, 1u);        // W_enc dZ_lo
+                                ptx::mma_ts(vcol, gcol + 2 * UNIT + k * 16 + 8, zmn + (uint64_t)(k * G::RB), idescO, 1u);    // W_enc lo x dZ_hi
                             }
                         }
                     }
@@ -743,10 +743,10 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // sweep 2: dS^T and W_enc^T of every unit, handed to the issuing warp
             auto unit2 = [&](auto masked, int u) {
                 constexpr bool kMasked = decltype(masked)::value;
-                uint32_t pwl[UNIT / 2];                                             // lo halves of W_enc, stored last
+                uint32_t pwl[4];                                    // lo halves of W_enc of an even quarter, kept for one quarter
 #pragma unroll
                 for (int qd = 0; qd < UNIT / 8; ++qd) {
-                    uint32_t s[8], av[8], cv[8], pk[4], pl[4], pw[4];
+                    uint32_t s[8], av[8], cv[8], pk[4], pl[4], pw[4], pwo[4];
                     ptx::tmem_ld8(gcol + qd * 8, s);
                     ptx::tmem_ld8(gcol + UNIT + qd * 8, av);
                     ptx::tmem_ld8(gcol + 2 * UNIT + qd * 8, cv);
@@ -769,15 +769,22 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         pl[k] = ptx::pack_bf16(ds.x - __uint_as_float(hi << 16), ds.y - __uint_as_float(hi & 0xffff0000u));
                         const uint32_t wh = ptx::pack_bf16(pe.x, pe.y);
                         pw[k] = wh;
-                        pwl[qd * 4 + k] = ptx::pack_bf16(pe.x - __uint_as_float(wh << 16), pe.y - __uint_as_float(wh & 0xffff0000u));
+                        pwo[k] = ptx::pack_bf16(pe.x - __uint_as_float(wh << 16), pe.y - __uint_as_float(wh & 0xffff0000u));
                     }
-                    // packed results over columns this thread has already read: dS hi over S, dS lo over A, W_enc over C
+                    // Packed results over columns this thread has already read: dS hi over S, dS lo over A.  W_enc over
+                    // C, per 16 latents (two quarters): hi in the first 8 of their 16 columns, lo in the other 8 - which
+                    // the odd quarter has only just read, so the even quarter's lo waits in four registers.
                     ptx::tmem_st4(gcol + qd * 4, pk);
                     ptx::tmem_st4(gcol + UNIT + qd * 4, pl);
-                    ptx::tmem_st4(gcol + 2 * UNIT + qd * 4, pw);
+                    ptx::tmem_st4(gcol + 2 * UNIT + (qd >> 1) * 16 + (qd & 1) * 4, pw);
+                    if (qd & 1) {
+                        ptx::tmem_st4(gcol + 2 * UNIT + (qd >> 1) * 16 + 8, pwl);
+                        ptx::tmem_st4(gcol + 2 * UNIT + (qd >> 1) * 16 + 12, pwo);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) pwl[k] = pwo[k];
+                    }
                 }
-                // the upper half of the score columns is free once all of them have been read
-                if (UNIT == 32) ptx::tmem_st16(gcol + UNIT / 2, pwl); else ptx::tmem_st8(gcol + UNIT / 2, pwl);
             };
             for (int u = 0; ok && u < nu; ++u) {
                 if (!warp_wait(bar(S_FULL + g), cnt & 1, abort_flag, kErrBwdTok | 7)) { ok = false; break; }
