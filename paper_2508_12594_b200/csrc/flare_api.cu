@@ -203,7 +203,7 @@ int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
 constexpr float kLog2e = 1.4426950408889634f;
 
 // kDz: the backward's dZ form of the kernel (V is then dY, lse_dec the decode log-sum-exp rows, pm and pl unused).
-template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false>
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false>
 int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
                      const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
                      const float *lse_dec = nullptr) {
@@ -217,7 +217,7 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     const size_t smem = EncodeSmem<DG>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     EncodeTcArgs a;
@@ -228,7 +228,7 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -300,10 +300,9 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     return FLARE_OK;
 }
 
-template <int D, int DRT = 0, bool kPart = false>
-int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
-                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0 = 0, int mc = 0, float *Ypart = nullptr) {
-    if (mc == 0) mc = d->M;                                     // the launch's range of latents: [m0, m0 + mc)
+template <int D, int DRT, bool kPart, int kM>
+int launch_decode_tc_m(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart) {
     CUtensorMap tmK, tmQ;
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
@@ -312,7 +311,7 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     const size_t smem = DecodeSmem<D>::total(mc);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT, kPart>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT, kPart, kM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     DecodeTcArgs a;
@@ -328,9 +327,23 @@ int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
     dim3 grid((unsigned)per_head, d->H, d->B);
-    decode_tc_kernel<D, DRT, kPart><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
+    decode_tc_kernel<D, DRT, kPart, kM><<<grid, kTcThreads, smem, st>>>(tmK, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
+}
+
+// The launch's range of latents is [m0, m0 + mc) (mc = 0: all of them).  The sizes that the workloads use most have
+// forms of the kernel with the number of latents as a compile-time constant.
+template <int D, int DRT = 0, bool kPart = false>
+int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0 = 0, int mc = 0, float *Ypart = nullptr) {
+    if (mc == 0) mc = d->M;
+    if (mc == 256) return launch_decode_tc_m<D, DRT, kPart, 256>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 128) return launch_decode_tc_m<D, DRT, kPart, 128>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 64) return launch_decode_tc_m<D, DRT, kPart, 64>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 32) return launch_decode_tc_m<D, DRT, kPart, 32>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 512) return launch_decode_tc_m<D, DRT, kPart, 512>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    return launch_decode_tc_m<D, DRT, kPart, 0>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
 }
 
 template <typename T>
@@ -574,9 +587,16 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
         TcEncodePlan p = tc_encode_plan(d, di.sms);
         uint32_t *status = reinterpret_cast<uint32_t *>(base);
         // a caller that asks for lse_enc is saving Z for the backward: weights as two bf16 halves (see exp_chunk_hilo)
-#define FLARE_ENC(DD, PAIR, DRT)                                                                                         \
-    (lse_enc != nullptr ? launch_encode_tc<DD, PAIR, false, DRT, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st) \
-                        : launch_encode_tc<DD, PAIR, false, DRT, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st))
+#define FLARE_ENC2(DD, PAIR, DRT, MB)                                                                                     \
+    (lse_enc != nullptr ? launch_encode_tc<DD, PAIR, false, DRT, true, MB>(d, p, Q, K, V, mask, pm, pl, pacc, status, st) \
+                        : launch_encode_tc<DD, PAIR, false, DRT, false, MB>(d, p, Q, K, V, mask, pm, pl, pacc, status, st))
+        // A call with a key mask has padding in every tile and takes the form that tests every element (see
+        // encode_tc_kernel).  Without a mask only a last partial tile has padding and either form serves; which one
+        // is faster was measured (B200): the form without the element tests where a CTA holds two latent blocks
+        // (M > 128: 0.80 -> 0.68 ms on the million-point shape, 223 -> 201 us at N = 131072, M = 512), the other
+        // where two slots share one block (M <= 128: 4-5 % apart).
+        const bool mask_body = mask != nullptr || d->M <= kTile;
+#define FLARE_ENC(DD, PAIR, DRT) (mask_body ? FLARE_ENC2(DD, PAIR, DRT, true) : FLARE_ENC2(DD, PAIR, DRT, false))
         if (encode_head_pairs(d))
             rc = d->D == 16 ? FLARE_ENC(16, true, 0) : FLARE_ENC(32, true, 0);
         else
@@ -586,6 +606,7 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
                  : d->D == 32 ? FLARE_ENC(32, false, 0)
                               : FLARE_ENC(64, false, 0);
 #undef FLARE_ENC
+#undef FLARE_ENC2
     } else {
         SimtPlan p = simt_plan(d, di.sms);
         rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)

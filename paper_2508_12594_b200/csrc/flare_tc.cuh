@@ -183,32 +183,32 @@ __host__ __device__ constexpr int decode_y_cols(int D) { return D <= 32 ? 2 * D 
 // top column down in chunks of 32; a chunk's columns are free once read.  With a Y accumulator of `yc` columns,
 // the first yc/16 chunks free 2*yc columns, which take those chunks' packed weights (16 columns each, top
 // down) and, below them, Y; every later chunk's weights go to the bottom half of the chunk's own columns.
-__host__ __device__ inline int decode_y_alias_col(int len, int yc) { return len - 2 * yc; }
+__host__ __device__ constexpr int decode_y_alias_col(int len, int yc) { return len - 2 * yc; }
 // First column (within the range) of the packed weights of the chunk whose scores start at column `lo`.
-__host__ __device__ inline int decode_p_col(int len, int yc, int lo, bool alias) {
+__host__ __device__ constexpr int decode_p_col(int len, int yc, int lo, bool alias) {
     const int k = (len - 1 - lo) / 32;                         // chunk index counted from the top
     return (alias && k < yc / 16) ? len - 16 * (k + 1) : lo;
 }
 // Score columns per hand-over of weights to the value contraction: at most four per range and tile, and the
 // first covers the 2*yc columns that make room for Y.
-__host__ __device__ inline int decode_handover_cols(int len, int yc) {
+__host__ __device__ constexpr int decode_handover_cols(int len, int yc) {
     int u = ((len + 3) / 4 + 31) & ~31;
     if (u < 2 * yc) u = 2 * yc;
     return u < 32 ? 32 : u;
 }
 
-__host__ __device__ inline int decode_part_len(const DecodePlan &p, int M, int c) {
+__host__ __device__ constexpr int decode_part_len(const DecodePlan &p, int M, int c) {
     const int start = c * p.part_w;
     const int len = M - start < p.part_w ? M - start : p.part_w;
     return len > 0 ? len : 0;
 }
 
-inline DecodePlan make_decode_plan(int M, int D) {
+__host__ __device__ constexpr DecodePlan make_decode_plan(int M, int D) {
     const int yc = decode_y_cols(D);
     DecodePlan best{};
     int best_groups = 0;
     for (int cs = 1; cs <= 4; cs *= 2) {
-        DecodePlan p;
+        DecodePlan p{};
         p.cs = cs;
         p.part_w = ((M / 16 + cs - 1) / cs) * 16;
         if ((cs - 1) * p.part_w >= M) continue;                 // an empty column range
@@ -272,7 +272,10 @@ struct DecodeSmem {
 //
 // Narrow form (DRT = 8 or 4 with D = 16): the head is DRT wide in memory (see narrow_offset).  This is how head
 // widths below the smallest MMA K-step (16) run on the tensor cores.
-template <int D, int DRT = 0, bool kPart = false>
+//
+// kM: 0, or the number of latents of the launch as a compile-time constant (the plan, the column choreography and
+// the chunk loops then fold to constants; the common sizes have such forms).
+template <int D, int DRT = 0, bool kPart = false, int kM = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
     constexpr bool kHalf = DRT != 0;
@@ -281,7 +284,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     using SM = DecodeSmem<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int M = a.M;
+    const int M = kM ? kM : a.M;
     uint8_t *sK = smem + SM::k_off;
     uint8_t *sQ = smem + SM::q_off(M);
     uint8_t *sZ = smem + SM::z_off(M);
@@ -304,7 +307,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int t_end = (int)((long)a.tiles * (blockIdx.x + 1) / gridDim.x);
     const int ntiles = t_end - t_begin;
 
-    const DecodePlan pl = a.plan;
+    constexpr DecodePlan kPlan = make_decode_plan(kM ? kM : 16, D);
+    const DecodePlan pl = kM ? kPlan : a.plan;
     const int cs = pl.cs, nbuf = pl.nbuf, cb = pl.cb;
     constexpr int YC = decode_y_cols(D);
     constexpr bool kWide = YC == 2 * D;                         // one MMA over [Z_hi | Z_lo] (N = 2D) per 16 latents
@@ -670,11 +674,22 @@ struct EncodeSmem {
     __host__ __device__ static size_t bar_off() { return q_off() + (size_t)2 * kTile * G::RB; }
     static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 32 * sizeof(float);   // per softmax warp: 2 x 32 column addends
     __host__ __device__ static size_t col_off() { return bar_off() + 512; }
+    // score bias of padded tokens: per stage a [128 tokens, 16] bf16 tile, then one [128 latents, 16] tile of ones
+    static constexpr size_t kBiasTile = kTile * 32;
+    __host__ __device__ static size_t bias_off() { return (col_off() + kColBytes + 1023) & ~(size_t)1023; }
     __host__ __device__ static size_t total() {
-        size_t t = col_off() + kColBytes + 1024;
+        size_t t = bias_off() + (kEncStages + 1) * kBiasTile + 1024;
         return t < kTcMinSmem ? kTcMinSmem : t;
     }
 };
+
+// Padding in encode.  A token that takes no part in the softmax (masked, or beyond N in the last tile) gets the
+// score kMaskedScore instead of a test per element: one more MMA k-step adds ones[latent] x bias[token] to the
+// tile's scores, with bias = kMaskedScore or 0 (exactly representable, so the scores of valid tokens do not
+// change).  Such a score never wins a maximum against a valid one and its weight 2^(score - max) is exactly 0.
+// A row that has seen no valid token yet has a running maximum at or below kDeadBelow and is treated as empty.
+constexpr float kMaskedScore = -1.0e30f;
+constexpr float kDeadBelow = -1.0e29f;
 
 // Encode, split over N.  grid = (splits, H * pairs, B).  A CTA owns up to two blocks of 128 latents of head h
 // ("slots", one TMEM score buffer each) and a contiguous range of token tiles.  With M <= 128 the two slots
@@ -701,7 +716,11 @@ struct EncodeSmem {
 // columns outside the head's (weights times the neighbours' values) are dropped.
 //
 // kHiLo: the weights go to the value contraction as two bf16 halves (see exp_chunk_hilo), as in the dZ form.
-template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false>
+//
+// kMaskBody: padded tokens are handled by a second form of the unit body that tests every element (the form for
+// calls with a key mask, where every tile has padding); without it they are handled in the scores (kMaskedScore),
+// which costs a bias tile and one more MMA per unit of the tiles that have padding, and nothing elsewhere.
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
@@ -751,7 +770,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
             ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? 128u
-                                   : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users : 1u);
+                                   : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users
+                                   : (i >= KV_FULL && i < KV_FULL + kEncStages) ? 2u : 1u);   // the TMA loads, the bias tile
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
@@ -762,6 +782,15 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // latent rows beyond M are zero so their (discarded) lanes stay finite
     for (int i = threadIdx.x; i < (2 * kTile - rows_here) * (G::RB / 16); i += kTcThreads)
         reinterpret_cast<uint4 *>(sQ + (size_t)rows_here * G::RB)[i] = make_uint4(0, 0, 0, 0);
+    uint8_t *sBias = smem + SM::bias_off();                     // [stage] bias tiles, then the tile of ones
+    if (!kDz) {
+        using GB = TileGeom<16>;
+        uint8_t *ones = sBias + (size_t)kEncStages * SM::kBiasTile;
+        for (int r = threadIdx.x; r < kTile; r += kTcThreads) {   // row r = [1, 0, ..., 0]: the first 16-byte chunk, swizzled
+            reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r)] = make_uint4(0x00003F80u, 0, 0, 0);
+            reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r) ^ 1] = make_uint4(0, 0, 0, 0);
+        }
+    }
     if (kPair) {
         // block-diagonal A operand: row r < 64 = [Q[h][r] | 0], row 64 + r = [0 | Q[h+1][r]], 16-byte chunks swizzled
         __syncthreads();
@@ -800,13 +829,33 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int r = 0; r < rows_here; r += 16)
                     ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
             }
-            for (int i = 0; i < nt; ++i) {
-                const int s = i % kEncStages;
-                if (!ptx::mbar_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
+        }
+        // The whole warp walks the tiles: lane 0 waits for the stage and issues the loads; for a tile with padding
+        // (masked tokens, or tokens beyond N) every lane first writes four rows of the stage's bias tile.
+        for (int i = 0; i < nt; ++i) {
+            const int s = i % kEncStages, t = t_begin + i;
+            if (!warp_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
+            const bool plain = kDz || kMaskBody || (a.key_mask == nullptr && (t + 1) * kTile <= a.N);
+            if (!plain) {
+                using GB = TileGeom<16>;
+                uint8_t *bt = sBias + (size_t)s * SM::kBiasTile;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int r = lane * 4 + k, n = t * kTile + r;
+                    const bool valid = n < a.N && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0);
+                    const uint32_t first = valid ? 0u : (uint32_t)__bfloat16_as_ushort(__float2bfloat16(kMaskedScore));
+                    reinterpret_cast<uint4 *>(bt + (size_t)r * GB::RB)[GB::swz(r)] = make_uint4(first, 0, 0, 0);
+                    reinterpret_cast<uint4 *>(bt + (size_t)r * GB::RB)[GB::swz(r) ^ 1] = make_uint4(0, 0, 0, 0);
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+            }
+            if (lane == 0) {
+                ptx::mbar_arrive(bar(KV_FULL + s));             // the bias tile (or none needed)
                 ptx::mbar_arrive_expect_tx(bar(KV_FULL + s), 2 * G::TILE_BYTES);
                 uint8_t *dst = sKV + (size_t)s * 2 * G::TILE_BYTES;
-                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(KV_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
-                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(KV_FULL + s), h * DR - off, t * kTile, b);
+                ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR - off, t * kTile, b);
             }
         }
     } else if (warp < kFirstSoftmaxWarp) {
@@ -837,6 +886,15 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                        (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
 #pragma unroll
                 for (int k = 0; k < DG / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                const int tile = t_begin + t_s;
+                if (!kDz && !kMaskBody && !(a.key_mask == nullptr && (tile + 1) * kTile <= a.N)) {
+                    // scores += ones x bias: padded tokens drop to kMaskedScore (see there)
+                    using GB = TileGeom<16>;
+                    const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)kEncStages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
+                    const uint64_t bdesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)s * SM::kBiasTile), 16, GB::SBO, GB::SWZ) +
+                                           (uint64_t)((c * HALF + w * UNIT) * GB::RB / 16);
+                    ptx::mma_ss(gcol + w * UNIT, odesc, bdesc, idescS, 1u);
+                }
                 ptx::mma_commit(bar(S_FULL + 2 * g + w));
                 if (w == 1) t_s += t_step;
                 return true;
@@ -942,7 +1000,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
             }
             m_run = m_new;
-            const bool dead = (m_run == -INFINITY);             // no valid token yet: all weights are zero
+            const bool dead = m_run < kDeadBelow;               // no valid token yet: all weights are zero
             const float neg = dead ? 0.f : -m_run * a.sl2;
             const float2 negp = make_float2(neg, neg);
             uint32_t pk[16];
@@ -964,10 +1022,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (j < nslots) {
             for (int q = j; ok && q < nq; q += nslots) {
                 const int t = t_begin + (alternate ? q : q / nslots);
-                const bool plain = a.key_mask == nullptr && (t + 1) * kTile <= a.N;   // warp-uniform
+                const bool plain = !kMaskBody || (a.key_mask == nullptr && (t + 1) * kTile <= a.N);   // warp-uniform
 #pragma unroll 1
-                for (int w = 0; ok && w < 2; ++w)               // the half's two units, on alternating buffers
-                    ok = kDz ? unit_dz(t, w) : plain ? unit(std::false_type{}, t, w) : unit(std::true_type{}, t, w);
+                for (int w = 0; ok && w < 2; ++w) {             // the half's two units, on alternating buffers
+                    if (kDz) ok = unit_dz(t, w);
+                    else if (kMaskBody && !plain) ok = unit(std::true_type{}, t, w);
+                    else ok = unit(std::false_type{}, t, w);    // (without kMaskBody padding is in the scores already)
+                }
             }
         }
         // write this group's partial (running max in natural-log units, sum, un-normalised rows)
@@ -992,7 +1053,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);
             const size_t prow = (size_t)part * rows + ((size_t)b * a.H + h + second) * M + m;
             if (!kDz) {
-                a.part_m[prow] = (m_run == -INFINITY) ? -INFINITY : m_run * a.scale;
+                a.part_m[prow] = (m_run < kDeadBelow) ? -INFINITY : m_run * a.scale;
                 a.part_l[prow] = l2.x + l2.y;
             }
             float4 *dst = reinterpret_cast<float4 *>(a.part_acc + prow * DR);
