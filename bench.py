@@ -32,8 +32,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) of one launch of each main kernel on the full mesh3d_1m workload, from the ncu captures
 # summarised under profiles/ (taken on a 262,144-token slice and scaled by 4: traffic is proportional to N).
 # Valid for the kernels as profiled; set to None when a kernel changes until the capture is redone.
-NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.321152e6 + 3.520256e6),
-               ("mesh3d_1m", "decode"): 4 * (67.362816e6 + 29.085184e6)}
+NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.330112e6 + 3.916544e6),
+               ("mesh3d_1m", "decode"): 4 * (68.004608e6 + 30.838016e6)}
 
 
 def get_workload(name: str) -> workloads.Workload:
