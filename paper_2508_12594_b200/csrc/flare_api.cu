@@ -263,12 +263,11 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     return FLARE_OK;
 }
 
-template <int D, int DRT = 0, int kMode = 0>
-int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
+template <int D, int DRT, int kMode, int kM>
+int launch_bwd_token_tc_m(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
                         const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
                         const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st,
-                        int m0 = 0, int mc = 0, float *kvacc = nullptr) {
-    if (mc == 0) mc = d->M;                                     // the launch's range of latents: [m0, m0 + mc)
+                        int m0, int mc, float *kvacc) {
     CUtensorMap tmK, tmV, tmG, tmQ;
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
@@ -282,7 +281,7 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     const size_t smem = BwdTokSmem<D>::total(a.stages, mc);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT, kMode, kM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
@@ -295,9 +294,26 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
     long per_head = sms / ((long)d->B * d->H);
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
-    bwd_token_tc_kernel<D, DRT, kMode><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_token_tc_kernel<D, DRT, kMode, kM><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
+}
+
+// The launch's range of latents is [m0, m0 + mc) (mc = 0: all of them); common sizes have forms of the kernel with
+// the number of latents as a compile-time constant.
+template <int D, int DRT = 0, int kMode = 0>
+int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
+                        const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
+                        const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st,
+                        int m0 = 0, int mc = 0, float *kvacc = nullptr) {
+    if (mc == 0) mc = d->M;
+#define FLARE_TOK(MM) launch_bwd_token_tc_m<D, DRT, kMode, MM>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd, status, st, m0, mc, kvacc)
+    if (mc == 256) return FLARE_TOK(256);
+    if (mc == 128) return FLARE_TOK(128);
+    if (mc == 64) return FLARE_TOK(64);
+    if (mc == 512) return FLARE_TOK(512);
+    return FLARE_TOK(0);
+#undef FLARE_TOK
 }
 
 template <int D, int DRT, bool kPart, int kM>

@@ -429,7 +429,8 @@ struct BwdTokSmem {
 // grid = (CTAs per head, H, B); a CTA takes the token tiles blockIdx.x, blockIdx.x + gridDim.x, ...
 // DRT = 8 or 4 (with D = 16): the narrow form (head DRT wide in memory; only the head's columns of the rows of dK
 // and dV are kept).
-template <int D, int DRT = 0, int kMode = 0>
+// kM: 0, or the number of latents of the launch as a compile-time constant.
+template <int D, int DRT = 0, int kMode = 0, int kM = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdTokTcArgs a) {
@@ -441,7 +442,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int M = a.M, MU = SM::padded_m(M), stages = a.stages;
+    const int M = kM ? kM : a.M, MU = SM::padded_m(M), stages = a.stages;
     uint8_t *sQ = smem + SM::lat_off(stages, M, 0);
     float *cst = reinterpret_cast<float *>(smem + SM::cst_off(stages, M));      // [MU] -lse_enc (log2 units), [MU] -de
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off(stages, M));
