@@ -233,8 +233,8 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     return FLARE_OK;
 }
 
-template <int D, int DRT = 0>
-int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
+template <int D, int DRT, bool kPadded>
+int launch_bwd_dq_tc_p(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
                      const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
                      const float *lse_dec, const float *dd, float *part, uint32_t *status, cudaStream_t st) {
     CUtensorMap tmK, tmV, tmG, tmQ;
@@ -247,7 +247,7 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     const size_t smem = BwdDqSmem<D>::total();
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_tc_kernel<D, DRT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_tc_kernel<D, DRT, kPadded>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     BwdDqTcArgs a;
@@ -258,12 +258,22 @@ int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, d->H * p.pairs, d->B);
-    bwd_dq_tc_kernel<D, DRT><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_dq_tc_kernel<D, DRT, kPadded><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 
-template <int D, int DRT, int kMode, int kM>
+template <int D, int DRT = 0>
+int launch_bwd_dq_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
+                     const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
+                     const float *lse_dec, const float *dd, float *part, uint32_t *status, cudaStream_t st) {
+    // padded tokens: a key mask, or a last partial tile
+    if (mask != nullptr || d->N % kTile != 0)
+        return launch_bwd_dq_tc_p<D, DRT, true>(d, p, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part, status, st);
+    return launch_bwd_dq_tc_p<D, DRT, false>(d, p, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part, status, st);
+}
+
+template <int D, int DRT, int kMode, int kM, bool kPadded>
 int launch_bwd_token_tc_m(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const void *dY,
                         const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
                         const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st,
@@ -281,7 +291,7 @@ int launch_bwd_token_tc_m(const flare_desc_t *d, int sms, const void *Q, const v
     const size_t smem = BwdTokSmem<D>::total(a.stages, mc);
     static bool attr_set = false;
     if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT, kMode, kM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT, kMode, kM, kPadded>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
@@ -294,7 +304,7 @@ int launch_bwd_token_tc_m(const flare_desc_t *d, int sms, const void *Q, const v
     long per_head = sms / ((long)d->B * d->H);
     if (per_head < 1) per_head = 1;
     if (per_head > a.tiles) per_head = a.tiles;
-    bwd_token_tc_kernel<D, DRT, kMode, kM><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_token_tc_kernel<D, DRT, kMode, kM, kPadded><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -307,7 +317,12 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
                         const float *lse_dec, void *dK, void *dV, float *dd, uint32_t *status, cudaStream_t st,
                         int m0 = 0, int mc = 0, float *kvacc = nullptr) {
     if (mc == 0) mc = d->M;
-#define FLARE_TOK(MM) launch_bwd_token_tc_m<D, DRT, kMode, MM>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd, status, st, m0, mc, kvacc)
+    const bool padded = mask != nullptr || d->N % kTile != 0;   // a key mask, or a last partial tile
+#define FLARE_TOK(MM)                                                                                                     \
+    (padded ? launch_bwd_token_tc_m<D, DRT, kMode, MM, true>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd, \
+                                                            status, st, m0, mc, kvacc)                                   \
+            : launch_bwd_token_tc_m<D, DRT, kMode, MM, false>(d, sms, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dK, dV, dd, \
+                                                             status, st, m0, mc, kvacc))
     if (mc == 256) return FLARE_TOK(256);
     if (mc == 128) return FLARE_TOK(128);
     if (mc == 64) return FLARE_TOK(64);

@@ -51,7 +51,9 @@ struct BwdDqSmem {
 // grid = (splits, H * pairs, B), as the encode kernel.  DRT = 8 or 4 (with D = 16): the narrow form of the forward
 // kernels (the head is DRT wide in memory; token tiles carry the neighbouring heads' features beside the head's
 // own, every latent operand zeros there, and the other columns of the partial dQ are dropped).
-template <int D, int DRT = 0>
+// kPadded: the launch has padded tokens (a key mask, or N not a multiple of the tile); without it the unit body that
+// tests validity is not compiled in.
+template <int D, int DRT = 0, bool kPadded = true>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdDqTcArgs a) {
@@ -331,7 +333,8 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll 1
                 for (int w = 0; ok && w < UPH; ++w) {
                     const uint32_t wv = ((w < 2 ? wv0 : wv1) >> ((w & 1) * UNIT)) & 0xffffu;
-                    ok = plain ? unit(std::false_type{}, w, wv) : unit(std::true_type{}, w, wv);
+                    if (kPadded && !plain) ok = unit(std::true_type{}, w, wv);
+                    else ok = unit(std::false_type{}, w, wv);
                 }
             }
         }
@@ -430,7 +433,8 @@ struct BwdTokSmem {
 // DRT = 8 or 4 (with D = 16): the narrow form (head DRT wide in memory; only the head's columns of the rows of dK
 // and dV are kept).
 // kM: 0, or the number of latents of the launch as a compile-time constant.
-template <int D, int DRT = 0, int kMode = 0, int kM = 0>
+// kPadded: as in the dQ kernel.
+template <int D, int DRT = 0, int kMode = 0, int kM = 0, bool kPadded = true>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdTokTcArgs a) {
@@ -791,7 +795,7 @@ bwd_token_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 if (!warp_wait(bar(S_FULL + g), cnt & 1, abort_flag, kErrBwdTok | 7)) { ok = false; break; }
                 ++cnt;
                 ptx::tc_fence_after();
-                if (plain) unit2(std::false_type{}, u); else unit2(std::true_type{}, u);
+                if (kPadded && !plain) unit2(std::true_type{}, u); else unit2(std::false_type{}, u);
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
                 ptx::mbar_arrive(bar(P_FULL + g));
