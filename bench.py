@@ -133,6 +133,17 @@ def whole_job_value(w, world: int, ms_step: float) -> float:
     return world * w.tokens / (ms_step / 1e3)
 
 
+def self_launch(n: int):
+    """`python bench.py --gpus N` outside a launcher: start the N replicas (one process per GPU) and relay rank 0's line."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.run(cmd).returncode)
+
+
 def run_reference(args, w):
     """The reference arm: the oracle on the host cores, each step a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -175,6 +186,8 @@ def main():
     w = get_workload(args.workload)
     if args.tokens > 0:
         w = w.with_(N=args.tokens, name=f"{w.name}@N={args.tokens}")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return self_launch(args.gpus)
     if args.impl == "reference":
         return run_reference(args, w)
     if args.warmup < 3:
@@ -284,7 +297,9 @@ def main():
         flare.flare_check(wsb)
         fb_ms = sum(a.elapsed_time(b) for a, b in pairs) / nb
         fwd_bwd = {"ms_per_step": fb_ms, "value": w.tokens / (fb_ms / 1e3), "unit": "tokens/s", "steps": nb,
-                   "gpu_launches_per_step": 10, "note": "per GPU; forward with saved statistics, then backward"}
+                   "gpu_launches_per_step": flare.flare_launch_count(desc, flare.OP_FORWARD) +
+                   flare.flare_launch_count(desc, flare.OP_BACKWARD),
+                   "note": "per GPU; forward with saved statistics, then backward"}
         del dYt, dK, dV, wsb
     if w.dtype == "bf16" and w.M > 512:
         # flare_decode has no workspace and runs more than 512 latents on the CUDA cores; inside flare_forward the
@@ -304,7 +319,8 @@ def main():
         if dist is not None:
             dist.destroy_process_group()
         return
-    finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist, fwd_bwd)
+    launches = args.steps * flare.flare_launch_count(desc, flare.OP_FORWARD)
+    finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist, fwd_bwd, launches)
 
 
 def run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V, mask, tensor_bytes, e):
@@ -329,7 +345,8 @@ def run_e2e(args, w, inp, flare, desc, ws, stream, barrier, dist, world, Q, K, V
             "d2h_bytes_per_step": tensor_bytes, "ms_per_step": e2e_ms}
 
 
-def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist, fwd_bwd=None):
+def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_bytes, e, l2_note, dist, fwd_bwd=None,
+           launches=0):
     peaks, peak_kind = load_peaks()
     # Roofline of the slower main kernel.  Per stage and head the contraction work is 4*N*M*D FLOP (scores and
     # value contraction); the bytes are K and V read (encode) or K read and Y written (decode), plus Q_lat.
@@ -362,7 +379,7 @@ def finish(args, w, inp, world, ms_step, value, stage_ms, clocks, e2e, tensor_by
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "M": w.M, "D": w.D, "scale": w.scale,
                    "l2": l2_note, "parallelism": f"replicas x{world}"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roof,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof,
     }
     if fwd_bwd is not None:
         out["fwd_bwd"] = fwd_bwd

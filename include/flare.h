@@ -89,6 +89,12 @@ size_t flare_workspace_bytes(const flare_desc_t *desc, int op);
 int flare_encode_partials(const flare_desc_t *desc);
 
 /*
+ * Number of kernels one call of the given operation launches for `desc` on the current device (0 for an invalid
+ * descriptor): e.g. encode, merge and decode for a forward; more where latents are worked off in ranges.
+ */
+int flare_launch_count(const flare_desc_t *desc, int op);
+
+/*
  * Encode (Section 3.2, encode equation; per-latent sum of the design-principles appendix):
  * Z and, if lse_enc != NULL, lse_enc.  Asking for lse_enc marks a forward whose Z will be differentiated through:
  * for bfloat16 inputs the softmax weights then enter the value contraction as two bfloat16 halves (Z within about
@@ -174,9 +180,23 @@ int flare_encode_static_scratch(const flare_desc_t *desc, const void *Q_lat, con
 /*
  * After the stream has been synchronised: FLARE_OK, or FLARE_ERR_TIMEOUT if a kernel of the last call that
  * used `workspace` gave up on a bounded wait (its outputs are then undefined).  Reads one word from the
- * workspace with a blocking copy.
+ * workspace with a blocking copy.  workspace = NULL means the built-in scratch array of
+ * flare_encode_static_scratch on the current device.  (flare_decode takes no workspace: a wait that gives up
+ * there is not reported; use flare_forward, or the workspace of a following call, where that matters.)
  */
 int flare_check(const void *workspace, flare_stream_t stream);
+
+/*
+ * Self-test of the bounded device-side waits (the paper has no counterpart).  Every wait inside the kernels
+ * (on a TMA load, on a tensor-core result) gives up after a time budget, records a code in the first word of
+ * the workspace and lets the kernel finish normally, so that a fault in the pipeline shows up as
+ * FLARE_ERR_TIMEOUT from flare_check instead of a hung GPU.  This call runs that mechanism in isolation: a
+ * one-block kernel waits for `budget_ns` nanoseconds (clamped to [1 us, 0.1 s]) on a barrier that nothing will
+ * ever complete, gives up, and records its code exactly as the other kernels do; flare_check(workspace) must
+ * then report FLARE_ERR_TIMEOUT, and the next ordinary call on the same workspace clears it.
+ * workspace: at least 256 bytes of device memory.
+ */
+int flare_selftest_wait(void *workspace, uint64_t budget_ns, flare_stream_t stream);
 
 #ifdef __cplusplus
 }

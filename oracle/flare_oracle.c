@@ -200,9 +200,9 @@ void flare_oracle_mixing_matrices(int B, int H, int N, int M, int D, double scal
  * Z, Y, lse_enc, lse_dec are recomputed here from the inputs (the oracle keeps no state).
  * Outputs: dQ [H, M, D] (summed over the batch), dK, dV [B, N, H, D]; dZ_out [B, H, M, D] may be NULL.
  */
-void flare_oracle_backward(int B, int H, int N, int M, int D, double scale, const double *Q, const double *K,
-                           const double *V, const uint8_t *key_mask, const double *dY, double *dQ, double *dK,
-                           double *dV, double *dZ_out) {
+static void backward_impl(int B, int H, int N, int M, int D, double scale, const double *Q, const double *K,
+                          const double *V, const uint8_t *key_mask, const double *dY, const int64_t *rows,
+                          int64_t nrows, double *dQ, double *dK, double *dV, double *dZ_out) {
     size_t nZ = (size_t)B * H * M * D, nT = (size_t)B * N * H * D;
     double *Z = (double *)malloc(sizeof(double) * nZ);
     double *dZ = (double *)calloc(nZ, sizeof(double));
@@ -226,31 +226,34 @@ void flare_oracle_backward(int B, int H, int N, int M, int D, double scale, cons
                 }
             }
 
-    /* per token: dV_n, dK_n */
-#pragma omp parallel for collapse(2) schedule(static)
-    for (int b = 0; b < B; ++b)
-        for (int n = 0; n < N; ++n)
-            for (int h = 0; h < H; ++h) {
-                const double *k = K + IDX_T(b, n, h), *v = V + IDX_T(b, n, h);
-                const double *dy = dY + IDX_T(b, n, h), *y = Y + IDX_T(b, n, h);
-                double *dk = dK + IDX_T(b, n, h), *dv = dV + IDX_T(b, n, h);
-                int valid = !(key_mask && !key_mask[(size_t)b * N + n]);
-                double delta_d = dot(dy, y, D);
-                for (int d = 0; d < D; ++d) dk[d] = 0.0, dv[d] = 0.0;
-                for (int m = 0; m < M; ++m) {
-                    const double *q = Q + IDX_Q(h, m);
-                    const double *z = Z + IDX_Z(b, h, m), *dz = dZ + IDX_Z(b, h, m);
-                    double s = scale * dot(k, q, D);
-                    double wdec = exp(s - ld[((size_t)b * N + n) * H + h]);
-                    double lem = le[((size_t)b * H + h) * M + m];
-                    double wenc = (valid && lem != -INFINITY) ? exp(s - lem) : 0.0;
-                    double dS = wdec * (dot(dy, z, D) - delta_d) + wenc * (dot(dz, v, D) - dot(dz, z, D));
-                    for (int d = 0; d < D; ++d) {
-                        dv[d] += wenc * dz[d];
-                        dk[d] += scale * dS * q[d];
-                    }
+    /* per token: dV_n, dK_n.  Token i of the list is rows[i] = b*N + n, or token i itself without a list; its
+       gradient rows go to row i of dK and dV. */
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < nrows; ++i) {
+        int64_t flat = rows ? rows[i] : i;
+        int b = (int)(flat / N), n = (int)(flat % N);
+        for (int h = 0; h < H; ++h) {
+            const double *k = K + IDX_T(b, n, h), *v = V + IDX_T(b, n, h);
+            const double *dy = dY + IDX_T(b, n, h), *y = Y + IDX_T(b, n, h);
+            double *dk = dK + ((size_t)i * H + h) * D, *dv = dV + ((size_t)i * H + h) * D;
+            int valid = !(key_mask && !key_mask[(size_t)b * N + n]);
+            double delta_d = dot(dy, y, D);
+            for (int d = 0; d < D; ++d) dk[d] = 0.0, dv[d] = 0.0;
+            for (int m = 0; m < M; ++m) {
+                const double *q = Q + IDX_Q(h, m);
+                const double *z = Z + IDX_Z(b, h, m), *dz = dZ + IDX_Z(b, h, m);
+                double s = scale * dot(k, q, D);
+                double wdec = exp(s - ld[((size_t)b * N + n) * H + h]);
+                double lem = le[((size_t)b * H + h) * M + m];
+                double wenc = (valid && lem != -INFINITY) ? exp(s - lem) : 0.0;
+                double dS = wdec * (dot(dy, z, D) - delta_d) + wenc * (dot(dz, v, D) - dot(dz, z, D));
+                for (int d = 0; d < D; ++d) {
+                    dv[d] += wenc * dz[d];
+                    dk[d] += scale * dS * q[d];
                 }
             }
+        }
+    }
 
     /* dQ: a reduction over tokens per (b,h,m), then over the batch in index order */
 #pragma omp parallel for collapse(3) schedule(dynamic)
@@ -279,6 +282,24 @@ void flare_oracle_backward(int B, int H, int N, int M, int D, double scale, cons
         for (size_t i = 0; i < (size_t)H * M * D; ++i) dQ[i] += dQb[(size_t)b * H * M * D + i];
     if (dZ_out) memcpy(dZ_out, dZ, sizeof(double) * nZ);
     free(Z); free(dZ); free(Y); free(le); free(ld); free(dQb);
+}
+
+void flare_oracle_backward(int B, int H, int N, int M, int D, double scale, const double *Q, const double *K,
+                           const double *V, const uint8_t *key_mask, const double *dY, double *dQ, double *dK,
+                           double *dV, double *dZ_out) {
+    backward_impl(B, H, N, M, D, scale, Q, K, V, key_mask, dY, NULL, (int64_t)B * N, dQ, dK, dV, dZ_out);
+}
+
+/*
+ * The same backward with the per-token gradients evaluated only for a list of sampled tokens (rows[i] = b*N + n;
+ * dK_rows, dV_rows [nrows, H, D]).  The reductions over all tokens (Z, Y, the log-sum-exp rows, dZ, dQ) still run
+ * in full: a token's dK_n and dV_n depend on the other tokens only through them.  For problem sizes at which the
+ * per-token loop over every token would dominate the run time.
+ */
+void flare_oracle_backward_rows(int B, int H, int N, int M, int D, double scale, const double *Q, const double *K,
+                                const double *V, const uint8_t *key_mask, const double *dY, const int64_t *rows,
+                                int nrows, double *dQ, double *dK_rows, double *dV_rows, double *dZ_out) {
+    backward_impl(B, H, N, M, D, scale, Q, K, V, key_mask, dY, rows, nrows, dQ, dK_rows, dV_rows, dZ_out);
 }
 
 int flare_oracle_max_threads(void) {

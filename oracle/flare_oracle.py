@@ -137,3 +137,18 @@ def backward(Q, K, V, dY, key_mask=None, scale=1.0):
                                   dQ.ctypes.data_as(_dp), dK.ctypes.data_as(_dp), dV.ctypes.data_as(_dp),
                                   dZ.ctypes.data_as(_dp))
     return dict(dQ=dQ, dK=dK, dV=dV, dZ=dZ)
+
+
+def backward_rows(Q, K, V, dY, rows, key_mask=None, scale=1.0):
+    """The backward with dK and dV evaluated only for the token rows ``rows`` (flat indices b*N+n); the reductions
+    over all tokens (dQ, dZ) run in full.  Returns dict(dQ [H,M,D], dK_rows, dV_rows [len(rows),H,D], dZ)."""
+    B, H, N, M, D = _dims(Q, K)
+    Q, pq = _d(Q); K, pk = _d(K); V, pv = _d(V); dY, pdy = _d(dY)
+    mk, pm = _mask(key_mask, B, N)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    dQ = np.empty((H, M, D)); dZ = np.empty((B, H, M, D))
+    dK = np.empty((len(rows), H, D)); dV = np.empty((len(rows), H, D))
+    _load().flare_oracle_backward_rows(B, H, N, M, D, ctypes.c_double(scale), pq, pk, pv, pm, pdy,
+                                       rows.ctypes.data_as(_i64p), len(rows), dQ.ctypes.data_as(_dp),
+                                       dK.ctypes.data_as(_dp), dV.ctypes.data_as(_dp), dZ.ctypes.data_as(_dp))
+    return dict(dQ=dQ, dK_rows=dK, dV_rows=dV, dZ=dZ)

@@ -1,6 +1,7 @@
 // Host side of libflare: argument checks, launch plans, kernel launches.  See include/flare.h for the contract.
 #include "../../include/flare.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -31,33 +32,51 @@ int cuda_fail(cudaError_t e, const char *what) {
     } while (0)
 
 struct DeviceInfo {
-    int checked = 0;  // 0 = not yet, 1 = ok, -1 = wrong arch, -2 = no device
-    int sms = 148;
+    std::atomic<int> checked{0};  // 0 = not yet, 1 = ok, -1 = wrong arch, -2 = no device
+    std::atomic<int> sms{148};
 };
 DeviceInfo g_dev[64];
 
-// Properties of the current device (cached per ordinal).  Without a device the plan falls back to 148 SMs so
-// that size queries still answer.
-const DeviceInfo &device_info(int *ordinal_out = nullptr) {
-    static DeviceInfo none{-2, 148};
+// Properties of the current device (cached per ordinal; concurrent first calls write the same values).  Without
+// a device the plan falls back to 148 SMs so that size queries still answer.
+struct DeviceView {
+    int checked, sms;
+};
+DeviceView device_info(int *ordinal_out = nullptr) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
         cudaGetLastError();
-        return none;
+        return DeviceView{-2, 148};
     }
     if (ordinal_out) *ordinal_out = dev;
     DeviceInfo &d = g_dev[dev];
-    if (d.checked == 0) {
+    int checked = d.checked.load(std::memory_order_acquire);
+    if (checked == 0) {
         int major = 0, sms = 0;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
             cudaGetLastError();
-            return none;
+            return DeviceView{-2, 148};
         }
-        d.sms = sms > 0 ? sms : 148;
-        d.checked = (major == 10) ? 1 : -1;
+        d.sms.store(sms > 0 ? sms : 148, std::memory_order_relaxed);
+        checked = (major == 10) ? 1 : -1;
+        d.checked.store(checked, std::memory_order_release);
     }
-    return d;
+    return DeviceView{checked, d.sms.load(std::memory_order_relaxed)};
+}
+
+// The opt-in to more than 48 KB of dynamic shared memory is a property of (kernel, device): one bit per device
+// ordinal in a mask per kernel instantiation.  Setting it twice is harmless, so a race between host threads
+// only repeats the call.
+template <typename Kernel>
+int ensure_big_smem(Kernel kernel, std::atomic<uint64_t> &done, int bytes = 227 * 1024) {
+    int dev = 0;
+    FLARE_CUDA(cudaGetDevice(&dev));
+    const uint64_t bit = 1ull << (dev & 63);
+    if (done.load(std::memory_order_acquire) & bit) return FLARE_OK;
+    FLARE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done.fetch_or(bit, std::memory_order_release);
+    return FLARE_OK;
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -215,11 +234,8 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = EncodeSmem<DG>::total();
-    static bool attr_set = false;
-    if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
-    }
+    static std::atomic<uint64_t> smem_opt_in{0};
+    if (int rc_attr = ensure_big_smem(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody>, smem_opt_in, 227 * 1024)) return rc_attr;
     EncodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.lse_dec = lse_dec;
@@ -245,11 +261,8 @@ int launch_bwd_dq_tc_p(const flare_desc_t *d, const TcEncodePlan &p, const void 
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = BwdDqSmem<D>::total();
-    static bool attr_set = false;
-    if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_tc_kernel<D, DRT, kPadded>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
-    }
+    static std::atomic<uint64_t> smem_opt_in{0};
+    if (int rc_attr = ensure_big_smem(bwd_dq_tc_kernel<D, DRT, kPadded>, smem_opt_in, 227 * 1024)) return rc_attr;
     BwdDqTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.dZ = dZ; a.lse_enc = lse_enc; a.de = de; a.lse_dec = lse_dec; a.dd = dd;
@@ -289,11 +302,8 @@ int launch_bwd_token_tc_m(const flare_desc_t *d, int sms, const void *Q, const v
     a.stages = BwdTokSmem<D>::stages(mc);
     if (a.stages < 1) return FLARE_ERR_UNSUPPORTED;
     const size_t smem = BwdTokSmem<D>::total(a.stages, mc);
-    static bool attr_set = false;
-    if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(bwd_token_tc_kernel<D, DRT, kMode, kM, kPadded>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
-    }
+    static std::atomic<uint64_t> smem_opt_in{0};
+    if (int rc_attr = ensure_big_smem(bwd_token_tc_kernel<D, DRT, kMode, kM, kPadded>, smem_opt_in, 227 * 1024)) return rc_attr;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.dZ = dZ; a.lse_enc = lse_enc; a.de = de; a.lse_dec = lse_dec; a.key_mask = mask;
     a.dK = (__nv_bfloat16 *)dK; a.dV = (__nv_bfloat16 *)dV; a.dd = dd; a.status = status;
@@ -340,11 +350,8 @@ int launch_decode_tc_m(const flare_desc_t *d, int sms, const void *Q, const void
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = DecodeSmem<D>::total(mc);
-    static bool attr_set = false;
-    if (!attr_set) {
-        FLARE_CUDA(cudaFuncSetAttribute(decode_tc_kernel<D, DRT, kPart, kM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
-    }
+    static std::atomic<uint64_t> smem_opt_in{0};
+    if (int rc_attr = ensure_big_smem(decode_tc_kernel<D, DRT, kPart, kM>, smem_opt_in, 227 * 1024)) return rc_attr;
     DecodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.Y = (__nv_bfloat16 *)Y; a.lse_dec = lse_dec; a.status = status;
@@ -561,12 +568,8 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     }
     if (!dq_on_tc) {
         const size_t dyn = sizeof(float) * 3 * (size_t)pb.LM * (D + 1);
-        static bool attr_set = false;
-        if (!attr_set) {
-            FLARE_CUDA(cudaFuncSetAttribute(bwd_dq_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)(sizeof(float) * 3 * 64 * (D + 1))));
-            attr_set = true;
-        }
+        static std::atomic<uint64_t> smem_opt_in{0};
+        if (int rc_attr = ensure_big_smem(bwd_dq_simt_kernel<T, D>, smem_opt_in, (int)(sizeof(float) * 3 * 64 * (D + 1)))) return rc_attr;
         bwd_dq_simt_kernel<T, D><<<dim3(pb.splits, d->H, d->B), kBwdThreads, dyn, st>>>(
             (const T *)Q, (const T *)K, (const T *)V, mask, (const T *)dY, Z, dZ, de, dd, lse_enc, lse_dec, part, d->B, d->H,
             d->N, d->M, pb.LM, pb.chunk, d->scale);
@@ -593,7 +596,7 @@ int backward_simt(const flare_desc_t *d, int sms, const void *Q, const void *K, 
 }
 
 int require_device() {
-    const DeviceInfo &di = device_info();
+    const DeviceView di = device_info();
     if (di.checked == -2) {
         snprintf(g_cuda_error, sizeof(g_cuda_error), "no CUDA device");
         return FLARE_ERR_CUDA;
@@ -604,7 +607,7 @@ int require_device() {
 
 int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void *V, const uint8_t *mask, float *Z,
                 float *lse_enc, void *ws, cudaStream_t st) {
-    const DeviceInfo &di = device_info();
+    const DeviceView di = device_info();
     const long rows = (long)d->B * d->H * d->M;
     const int P = partials_for(d, di.sms);
     WorkspaceLayout w = make_layout(P, rows, d->D, false);
@@ -708,24 +711,41 @@ int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float
 // Scratch of flare_encode_static_scratch: part of the device image, shared by every call on the device.
 // In host code this name is only a handle for cudaGetSymbolAddress; kernels must be given the looked-up address.
 static __device__ __align__(256) unsigned char g_static_scratch[FLARE_STATIC_SCRATCH_BYTES];
-void *g_static_scratch_addr[64] = {};
+std::atomic<void *> g_static_scratch_addr[64];
 
 // Device address of g_static_scratch on the current device (looked up once per device, then cached).
 int static_scratch_address(void **out) {
     int dev = -1;
     FLARE_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return FLARE_ERR_UNSUPPORTED;
-    if (g_static_scratch_addr[dev] == nullptr) {
-        void *p = nullptr;
+    void *p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
         FLARE_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
         if (p == nullptr) {
             snprintf(g_cuda_error, sizeof(g_cuda_error), "cudaGetSymbolAddress returned a null address");
             return FLARE_ERR_CUDA;
         }
-        g_static_scratch_addr[dev] = p;
+        g_static_scratch_addr[dev].store(p, std::memory_order_release);
     }
-    *out = g_static_scratch_addr[dev];
+    *out = p;
     return FLARE_OK;
+}
+
+// Kernels one call of `op` launches (the memset of the workspace header is not a kernel).
+int launches_for(const flare_desc_t *d, int op, int sms) {
+    const int enc = 2;                                          // encode, merge
+    const int dec = decode_in_ranges(d) ? decode_ranges(d) + 1 : 1;   // ranges of latents and their combination
+    switch (op) {
+        case FLARE_OP_ENCODE: return enc;
+        case FLARE_OP_DECODE: return 1;                         // without a workspace there are no ranges
+        case FLARE_OP_FORWARD: return enc + dec;
+        case FLARE_OP_BACKWARD: {
+            (void)sms;
+            const int tok = token_in_ranges(d) ? 2 * ((d->M + token_range(d) - 1) / token_range(d)) : 1;
+            return 3 + tok + 2;                                 // dZ, its reduction, de; token kernel(s); dQ, its reduction
+        }
+        default: return 0;
+    }
 }
 
 }  // namespace
@@ -752,6 +772,11 @@ const char *flare_last_cuda_error(void) { return g_cuda_error; }
 int flare_encode_partials(const flare_desc_t *desc) {
     if (check_desc(desc) != FLARE_OK) return 0;
     return partials_for(desc, device_info().sms);
+}
+
+int flare_launch_count(const flare_desc_t *desc, int op) {
+    if (check_desc(desc) != FLARE_OK) return 0;
+    return launches_for(desc, op, device_info().sms);
 }
 
 size_t flare_workspace_bytes(const flare_desc_t *desc, int op) {
@@ -874,11 +899,29 @@ int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void 
 }
 
 int flare_check(const void *workspace, flare_stream_t stream) {
-    if (!workspace) return FLARE_ERR_INVALID_ARG;
+    void *builtin = nullptr;
+    if (!workspace) {                                           // the built-in scratch of flare_encode_static_scratch
+        const int rc = static_scratch_address(&builtin);
+        if (rc != FLARE_OK) return rc;
+        workspace = builtin;
+    }
     uint32_t words[2] = {0, 0};
     FLARE_CUDA(cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     FLARE_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
     return words[0] == 0 ? FLARE_OK : FLARE_ERR_TIMEOUT;
+}
+
+int flare_selftest_wait(void *workspace, uint64_t budget_ns, flare_stream_t stream) {
+    if (!workspace || !aligned16(workspace)) return FLARE_ERR_INVALID_ARG;
+    int rc = require_device();
+    if (rc != FLARE_OK) return rc;
+    if (budget_ns < 1000) budget_ns = 1000;
+    if (budget_ns > 100000000ull) budget_ns = 100000000ull;     // never more than a tenth of a second
+    cudaStream_t st = (cudaStream_t)stream;
+    FLARE_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, st));
+    selftest_wait_kernel<<<1, 32, 0, st>>>(static_cast<uint32_t *>(workspace), (unsigned long long)budget_ns);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
 }
 
 }  // extern "C"

@@ -61,9 +61,10 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 // Wait budget of one barrier wait, in nanoseconds of the global timer.
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;
 
-// Bounded wait.  Returns false if the barrier did not flip within the budget or if another thread of the
+// Bounded wait.  Returns false if the barrier did not flip within `budget_ns` or if another thread of the
 // block already gave up (*abort_flag != 0); in the first case it records `code` in *abort_flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t code) {
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t code,
+                                              uint64_t budget_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
@@ -71,12 +72,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0) {
             if (*abort_flag != 0) return false;
-            if (globaltimer_ns() - t0 > kWaitBudgetNs) {
+            if (globaltimer_ns() - t0 > budget_ns) {
                 *abort_flag = code;
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t code) {
+    return mbar_wait_for(bar, parity, abort_flag, code, kWaitBudgetNs);
 }
 
 // ---------------------------------------------------------------- fences

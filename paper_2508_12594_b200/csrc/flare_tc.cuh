@@ -38,7 +38,8 @@ constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode)
 constexpr size_t kTcMinSmem = 120 * 1024;  // request at least this much so that one CTA owns an SM (and its TMEM)
 
 // Error codes left in the workspace header by a wait that gave up.
-enum : uint32_t { kErrDecode = 0x100, kErrEncode = 0x200, kErrBwdDq = 0x300, kErrBwdTok = 0x400 };
+enum : uint32_t { kErrDecode = 0x100, kErrEncode = 0x200, kErrBwdDq = 0x300, kErrBwdTok = 0x400, kErrSelftest = 0x500,
+                  kErrSpectral = 0x600 };
 
 // Bounded wait whose outcome is the same for every lane of the warp, so that the warp-collective tensor-memory
 // instructions that follow are executed by all lanes or by none.
@@ -1075,6 +1076,23 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         ptx::tmem_dealloc(tm, NCOLS);
     }
     if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
+}
+
+// The bounded wait of the kernels above, on its own: one thread waits for at most `budget_ns` on a barrier phase
+// that nothing ever completes, then takes the same way out as a kernel whose wait gave up (code into the block's
+// abort flag, from there into the workspace header).  Lets a caller see FLARE_ERR_TIMEOUT without a hung kernel.
+__global__ void selftest_wait_kernel(uint32_t *status, unsigned long long budget_ns) {
+    __shared__ uint64_t bar_mem;
+    __shared__ uint32_t flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&bar_mem), 1);
+        flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) ptx::mbar_wait_for(ptx::smem_u32(&bar_mem), 0, &flag, kErrSelftest | 1, budget_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && flag != 0 && status != nullptr) atomicCAS(status, 0u, flag);
 }
 
 }  // namespace flare

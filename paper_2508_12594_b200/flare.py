@@ -51,6 +51,8 @@ _SIGNATURES = {
     "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 13 + [_sz, _vp]),
     "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
     "flare_check": (ctypes.c_int, [_vp, _vp]),
+    "flare_launch_count": (ctypes.c_int, [_dp, ctypes.c_int]),
+    "flare_selftest_wait": (ctypes.c_int, [_vp, ctypes.c_uint64, _vp]),
 }
 
 
@@ -208,7 +210,16 @@ def flare_forward_host(desc, hQ, hK, hV, hmask, hY, dQ, dK, dV, dmask, dY, works
 
 
 def flare_check(workspace, stream=None):
+    """workspace=None checks the built-in scratch array of flare_encode_static_scratch."""
     _raise(load().flare_check(_ptr(workspace, torch.uint8), _stream(stream)), "flare_check")
+
+
+def flare_launch_count(desc: FlareDesc, op: int) -> int:
+    return int(load().flare_launch_count(ctypes.byref(desc), op))
+
+
+def flare_selftest_wait(workspace, budget_ns: int, stream=None):
+    _raise(load().flare_selftest_wait(_ptr(workspace, torch.uint8), int(budget_ns), _stream(stream)), "flare_selftest_wait")
 
 
 def forward(Q, K, V, key_mask=None, scale=1.0, want_stats=False, stream=None):

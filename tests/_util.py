@@ -22,25 +22,34 @@ def bf16_round(x):
     return torch.from_numpy(np.asarray(x, dtype=np.float64)).float().bfloat16().double().numpy()
 
 
+# Which bound every stored-tensor comparison met: (what, bound, max|err|/RMS, (max|err| - one rounding)/RMS).
+# conftest.py writes the list to the file named by FLARE_PARITY_REPORT at the end of the session.
+BOUND_LOG = []
+
+
 def assert_stored_close(got, ref, dtype, what):
-    """The bound on a tensor that is stored in the call dtype.
+    """The bound on a tensor that is stored in the call dtype.  Returns "stated" or "stated+rounding".
 
     The stated bound is max|err| <= tol * RMS(ref).  For a bfloat16 tensor it cannot hold for entries larger than
     about 5 RMS whatever the kernel does: rounding the exact value to bfloat16 is an error of up to 2^-8 |ref|,
     which passes 2e-2 RMS at |ref| = 5.12 RMS (the mesh workloads have entries of 8 RMS and more; the oracle's own
     Y rounded to bfloat16 breaks the stated bound there, see test_oracle_pins.py).  So the stated bound is tried
     first, and where it fails the bound is the stated one plus exactly one rounding of the stored value:
-    |err| <= tol * RMS(ref) + 2^-8 |ref|, element by element."""
+    |err| <= tol * RMS(ref) + 2^-8 |ref|, element by element.  Which of the two a case needed is recorded."""
     tol = TOL[dtype]
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     rms = max(float(np.sqrt(np.mean(ref ** 2))), 1e-300)
     err = np.abs(got - ref)
-    if err.max() <= tol * rms:
-        return
-    assert dtype == "bf16", f"{what}: max|err|/RMS = {err.max() / rms:.3e} > {tol}"
-    excess = (err - 2.0 ** -8 * np.abs(ref)).max() / rms
+    plain = float(err.max()) / rms
+    if plain <= tol:
+        BOUND_LOG.append((what, "stated", plain, None))
+        return "stated"
+    assert dtype == "bf16", f"{what}: max|err|/RMS = {plain:.3e} > {tol}"
+    excess = float((err - 2.0 ** -8 * np.abs(ref)).max()) / rms
+    BOUND_LOG.append((what, "stated+rounding", plain, excess))
     assert excess <= tol, f"{what}: (max|err| - one bf16 rounding)/RMS = {excess:.3e} > {tol}"
+    return "stated+rounding"
 
 
 def to_np64(t):
@@ -51,9 +60,11 @@ def dev(t):
     return None if t is None else t.cuda()
 
 
-def gpu_forward(inp, scale=1.0, canary=False):
+def gpu_forward(inp, scale=1.0, canary=False, stats=True):
     """flare_forward on cuda:0.  With canary=True the outputs sit inside larger buffers whose margins must stay
-    untouched (checked here).  Returns numpy float64 dict(Y, Z, lse_enc, lse_dec)."""
+    untouched (checked here).  stats=False is the inference call the benchmark times: Z is asked for, the two
+    log-sum-exp outputs are NULL (which selects other forms of the kernels).  Returns numpy float64
+    dict(Y, Z, lse_enc, lse_dec), the last two None without stats."""
     Q, K, V, mask = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask)
     desc = flare.make_desc(Q, K, scale)
     B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
@@ -71,13 +82,15 @@ def gpu_forward(inp, scale=1.0, canary=False):
     ldb, ld = padded((B, N, H), torch.float32, 777.0)
     if pad % 8 != 0:
         raise AssertionError("canary margin must keep 16-byte alignment")
-    flare.flare_forward(desc, Q, K, V, mask, Y, Z, le, ld, ws)
+    flare.flare_forward(desc, Q, K, V, mask, Y, Z, le if stats else None, ld if stats else None, ws)
     torch.cuda.synchronize()
     flare.flare_check(ws)
     if canary:
         for buf in (Yb, Zb, leb, ldb):
             assert (buf[:pad] == 777.0).all() and (buf[-pad:] == 777.0).all(), "write outside an output buffer"
-    return dict(Y=to_np64(Y), Z=to_np64(Z), lse_enc=to_np64(le), lse_dec=to_np64(ld))
+    if not stats:
+        assert (le == 777.0).all() and (ld == 777.0).all(), "an output that was not asked for was written"
+    return dict(Y=to_np64(Y), Z=to_np64(Z), lse_enc=to_np64(le) if stats else None, lse_dec=to_np64(ld) if stats else None)
 
 
 def oracle_forward(oracle, inp, scale=1.0):
@@ -91,6 +104,8 @@ def assert_forward_close(got, ref, dtype, what=""):
     assert e <= tol, f"{what} Z: max|err|/RMS = {e:.3e} > {tol}"
     assert_stored_close(got["Y"], ref["Y"], dtype, f"{what} Y")
     for name in ("lse_enc", "lse_dec"):
+        if got[name] is None:
+            continue
         fin = np.isfinite(ref[name])
         assert np.array_equal(np.isneginf(got[name]), np.isneginf(ref[name])), f"{what} {name}: -inf pattern"
         if fin.any():

@@ -27,3 +27,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """Write which bound every stored-tensor comparison met (see tests/_util.py) where FLARE_PARITY_REPORT names a file."""
+    path = os.environ.get("FLARE_PARITY_REPORT")
+    if not path:
+        return
+    from tests import _util
+    with open(path, "w") as f:
+        for what, bound, plain, excess in _util.BOUND_LOG:
+            f.write(f"{what}\t{bound}\t{plain:.3e}\t{'' if excess is None else format(excess, '.3e')}\n")

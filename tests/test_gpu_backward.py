@@ -2,7 +2,7 @@
 
 The gradients are those of sum(Y * dY).  Tolerance per tensor (dQ_lat, dK, dV):
     |got - ref| <= tol * RMS(ref) + store_ulp * |ref|     element by element,
-tol = 2e-2 for bfloat16 inputs (the forward's bound) and 1e-4 for float32 (a gradient entry is a sum of M or N
+tol = 2e-2 for bfloat16 inputs (the forward's bound) and 2e-5 for float32 (a gradient entry is a sum of M or N
 signed terms dS * q, each carrying the float32 rounding of an exponential and of two D-term dot products that
 nearly cancel, dY.Z_m - dY.Y, so its error relative to the tensor's RMS is a few 1e-6 and grows with sqrt(M)).
 store_ulp = 2^-8 for dK and dV stored as bfloat16, 0 otherwise: gradients are heavy-tailed (max/RMS of 20 to 60
@@ -17,11 +17,11 @@ import pytest
 import torch
 
 from paper_2508_12594_b200 import flare, workloads
-from tests._util import dev, rel_err, to_np64
+from tests._util import BOUND_LOG, dev, rel_err, to_np64
 
 pytestmark = pytest.mark.gpu
 
-GRAD_TOL = {"f32": 1e-4, "bf16": 2e-2}
+GRAD_TOL = {"f32": 2e-5, "bf16": 2e-2}
 
 
 def gpu_backward(inp, scale=1.0):
@@ -43,8 +43,11 @@ def assert_grads_close(got, ref, dtype, what, floor=None):
         if floor is not None:
             rms = max(rms, floor[name])
         store_ulp = 2.0 ** -8 if (dtype == "bf16" and name != "dQ") else 0.0
-        excess = np.abs(got[name] - ref[name]) - store_ulp * np.abs(ref[name])
+        err = np.abs(got[name] - ref[name])
+        excess = err - store_ulp * np.abs(ref[name])
         e = float(excess.max()) / max(rms, 1e-300)
+        plain = float(err.max()) / max(rms, 1e-300)
+        BOUND_LOG.append((f"{what} {name}", "stated" if plain <= GRAD_TOL[dtype] else "stated+rounding", plain, e))
         assert e <= GRAD_TOL[dtype], f"{what} {name}: (max|err| - ulp)/RMS = {e:.3e} > {GRAD_TOL[dtype]}"
 
 

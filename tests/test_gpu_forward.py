@@ -27,12 +27,19 @@ SCALED = [
 ]
 
 
+# stats: the training call (Z and both log-sum-exp outputs) or the inference call the benchmark times (Z only; the
+# library then runs other forms of its kernels: single bfloat16 encode weights, no statistics written)
+STATS = pytest.mark.parametrize("stats", [True, False], ids=["train", "infer"])
+
+
 @pytest.mark.parametrize("w", SCALED, ids=lambda w: w.name)
 @pytest.mark.parametrize("paper_scale", [True, False], ids=["s=1", "s=1/sqrtD"])
-def test_scaled_down_workloads(oracle, w, paper_scale):
+@STATS
+def test_scaled_down_workloads(oracle, w, paper_scale, stats):
     scale = 1.0 if paper_scale else w.D ** -0.5
     inp = workloads.make_inputs(w)
-    assert_forward_close(gpu_forward(inp, scale, canary=True), oracle_forward(oracle, inp, scale), w.dtype, w.name)
+    assert_forward_close(gpu_forward(inp, scale, canary=True, stats=stats), oracle_forward(oracle, inp, scale), w.dtype,
+                         f"{w.name} {'train' if stats else 'infer'}")
 
 
 EDGE = [
@@ -72,10 +79,12 @@ EDGE = [
 
 
 @pytest.mark.parametrize("case", EDGE, ids=lambda c: "B{}H{}N{}M{}D{}{}m{}".format(*c))
-def test_edge_shapes(oracle, case):
+@STATS
+def test_edge_shapes(oracle, case, stats):
     B, H, N, M, D, dtype, mf = case
     inp = workloads.make_random(B, H, N, M, D, dtype=dtype, seed=N + M, masked_fraction=mf, k_std=0.8)
-    assert_forward_close(gpu_forward(inp, canary=True), oracle_forward(oracle, inp), dtype, str(case))
+    assert_forward_close(gpu_forward(inp, canary=True, stats=stats), oracle_forward(oracle, inp), dtype,
+                         f"{case} {'train' if stats else 'infer'}")
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -175,9 +184,51 @@ def test_error_paths_on_device():
 
 
 @pytest.mark.parametrize("k_std", [3.0, 8.0])
-def test_large_scores(oracle, k_std):
+@STATS
+def test_large_scores(oracle, k_std, stats):
     """Scores up to +-170 at scale 1: the running maximum is subtracted before every exponential."""
     inp = workloads.make_random(1, 2, 700, 128, 16, dtype="bf16", seed=7, k_std=k_std)
-    got = gpu_forward(inp, canary=True)
+    got = gpu_forward(inp, canary=True, stats=stats)
     assert np.isfinite(got["Y"]).all() and np.isfinite(got["Z"]).all()
     assert_forward_close(got, oracle_forward(oracle, inp), "bf16", f"k_std={k_std}")
+
+
+@pytest.mark.parametrize("w", [workloads.CONFIGS["mesh2d"].with_(B=2, N=3001), workloads.CONFIGS["padded"].with_(B=3, N=1000)],
+                         ids=lambda w: w.name)
+def test_forward_from_host_buffers(oracle, w):
+    """flare_forward_host (the call behind the benchmark's end-to-end number): pinned host tensors in, a pinned host
+    tensor out, the device tensors being staging buffers only; the host result against the oracle."""
+    inp = workloads.make_inputs(w)
+    hQ, hK, hV = inp.Q.pin_memory(), inp.K.pin_memory(), inp.V.pin_memory()
+    hmask = None if inp.key_mask is None else inp.key_mask.pin_memory()
+    hY = torch.full_like(inp.K, 777.0).pin_memory()
+    desc = flare.make_desc(inp.Q, inp.K, w.scale)
+    dQ, dK, dV, dY = (torch.full_like(t, 555.0, device="cuda") for t in (inp.Q, inp.K, inp.V, inp.K))
+    dmask = None if hmask is None else torch.zeros_like(hmask, device="cuda")
+    ws = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    flare.flare_forward_host(desc, hQ, hK, hV, hmask, hY, dQ, dK, dV, dmask, dY, ws)
+    torch.cuda.synchronize()
+    flare.flare_check(ws)
+    ref = oracle_forward(oracle, inp, w.scale)
+    from tests._util import assert_stored_close
+    assert_stored_close(to_np64(hY), ref["Y"], w.dtype, f"{w.name} Y (host)")
+    assert torch.equal(hY, dY.cpu()) and torch.equal(dK.cpu(), inp.K)
+
+
+def test_bounded_wait_gives_up_and_reports(oracle):
+    """A device-side wait that nothing completes runs out of its time budget, the kernel ends normally, flare_check
+    reports FLARE_ERR_TIMEOUT, and the same workspace serves an ordinary forward afterwards."""
+    inp = workloads.make_random(1, 2, 300, 32, 16, dtype="bf16", seed=2)
+    Q, K, V = dev(inp.Q), dev(inp.K), dev(inp.V)
+    desc = flare.make_desc(Q, K)
+    ws = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    flare.flare_selftest_wait(ws, 1_000_000)                  # one millisecond
+    torch.cuda.synchronize()
+    with pytest.raises(flare.FlareError) as e:
+        flare.flare_check(ws)
+    assert e.value.status == flare.ERR_TIMEOUT
+    Y = torch.empty_like(K)
+    flare.flare_forward(desc, Q, K, V, None, Y, None, None, None, ws)
+    torch.cuda.synchronize()
+    flare.flare_check(ws)
+    assert rel_err(to_np64(Y), oracle_forward(oracle, inp)["Y"]) <= TOL["bf16"]

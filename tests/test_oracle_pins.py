@@ -248,17 +248,38 @@ def test_backward_value_gradient_sums(oracle):
     assert (g["dV"][mask == 0] == 0).all()
 
 
-def test_bf16_storage_alone_can_break_the_stated_bound(oracle):
-    """On the mesh workload the exact Y has entries of many RMS; rounding the oracle's own Y to bfloat16 is then by
-    itself an error above 2e-2 RMS(Y) at full size.  This is why the GPU tests allow one rounding of the stored
-    value on top of the stated bound where the stated bound fails."""
-    w = workloads.CONFIGS["mesh2d"].with_(B=1, N=16384)
+def test_backward_rows_matches_full(oracle):
+    """The sampled-rows backward is the full backward restricted to the listed tokens, bit for bit (dQ and dZ are
+    full reductions in both)."""
+    B, H, N, M, D = 2, 2, 41, 6, 4
+    inp = workloads.make_random(B, H, N, M, D, seed=43, masked_fraction=0.2, with_dy=True)
+    Q, K, V, mask, dY = _np(inp)
+    full = oracle.backward(Q, K, V, dY, key_mask=mask, scale=0.7)
+    rows = np.array([0, 3, 40, 41, 57, 81])
+    part = oracle.backward_rows(Q, K, V, dY, rows, key_mask=mask, scale=0.7)
+    np.testing.assert_array_equal(part["dQ"], full["dQ"])
+    np.testing.assert_array_equal(part["dZ"], full["dZ"])
+    np.testing.assert_array_equal(part["dK_rows"], full["dK"].reshape(B * N, H, D)[rows])
+    np.testing.assert_array_equal(part["dV_rows"], full["dV"].reshape(B * N, H, D)[rows])
+
+
+def test_bf16_storage_alone_breaks_the_stated_bound(oracle):
+    """On the 2-D mesh workload (one batch item at its full length) the exact Y has entries of many RMS, and rounding
+    the oracle's own Y to bfloat16 is by itself an error above 2e-2 RMS(Y): no kernel that stores bfloat16 can
+    meet the stated bound there.  This is why the GPU tests allow exactly one rounding of the stored value on top
+    of the stated bound where the stated bound fails (and report that they did)."""
+    w = workloads.CONFIGS["mesh2d"].with_(B=1)
     Q, K, V, _, _ = _np(workloads.make_inputs(w))
-    Y = oracle.forward(Q, K, V)["Y"]
+    Z, _ = oracle.encode(Q, K, V)
+    # the rows with the largest keys carry the largest outputs: decode those and a seeded sample for the RMS
+    knorm = np.abs(K).reshape(w.N, -1).max(axis=1)
+    rows = np.unique(np.concatenate([np.argsort(knorm)[-2048:], np.random.default_rng(0).choice(w.N, 8192, replace=False)]))
+    sample = np.random.default_rng(1).choice(w.N, 8192, replace=False)
+    Y = oracle.decode_rows(Q, K, Z, rows)
+    rms = np.sqrt(np.mean(oracle.decode_rows(Q, K, Z, sample) ** 2))
     Yb = torch.from_numpy(Y).float().bfloat16().double().numpy()
-    rms = np.sqrt(np.mean(Y ** 2))
     assert np.abs(Y).max() > 5.12 * rms
-    assert np.abs(Yb - Y).max() > 1.5e-2 * rms           # storage rounding alone takes most or all of the stated 2e-2
+    assert np.abs(Yb - Y).max() > 2e-2 * rms             # storage rounding alone exceeds the stated bound
     assert (np.abs(Yb - Y) <= 2.0 ** -8 * np.abs(Y)).all()
 
 

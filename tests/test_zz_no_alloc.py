@@ -7,6 +7,7 @@ flare_encode gives with a caller-allocated workspace -- twice in a row with diff
 array is shared and keeps the previous call's contents -- and that a problem too large for it is refused.
 Collected last on purpose: a failure here must not hide the other tests from a run that stops at the first.
 """
+import numpy as np
 import pytest
 import torch
 
@@ -32,18 +33,25 @@ def _encode_both(inp):
     return (Z, le), (Z_ref, le_ref)
 
 
-def test_static_scratch_encode_matches_encode_twice_in_a_row():
+def test_static_scratch_encode_matches_encode_twice_in_a_row(oracle):
     cases = [
         (workloads.CONFIGS["mesh3d_1m"].with_(N=20011), "bf16"),           # many splits: most of the partial slots
         (workloads.CONFIGS["padded"].with_(B=2, N=900), "bf16"),           # fewer, differently shaped partials + mask
         (workloads.CONFIGS["tiny"], "f32"),                                # the CUDA-core path
     ]
     for w, dtype in cases:
-        (Z, le), (Z_ref, le_ref) = _encode_both(workloads.make_inputs(w))
-        assert rel_err(to_np64(Z), to_np64(Z_ref)) <= TOL[dtype], w.name
-        fin = torch.isfinite(le_ref)
-        assert torch.equal(torch.isfinite(le), fin)
-        assert (le[fin] - le_ref[fin]).abs().max().item() <= (1e-4 if dtype == "f32" else 2e-2), w.name
+        inp = workloads.make_inputs(w)
+        (Z, le), (Z_ref, le_ref) = _encode_both(inp)
+        # the same kernels with the same split plan, only the scratch lives elsewhere: bit for bit the same
+        assert torch.equal(Z, Z_ref) and torch.equal(le, le_ref), w.name
+        flare.flare_check(None)                                            # no bounded wait gave up on the built-in array
+        # and both against the oracle, within the forward's bound
+        mk = None if inp.key_mask is None else inp.key_mask.numpy()
+        Zo, leo = oracle.encode(to_np64(inp.Q), to_np64(inp.K), to_np64(inp.V), key_mask=mk, scale=w.scale)
+        assert rel_err(to_np64(Z), Zo) <= TOL[dtype], w.name
+        fin = np.isfinite(leo)
+        assert np.array_equal(np.isfinite(to_np64(le)), fin)
+        assert np.abs(to_np64(le)[fin] - leo[fin]).max() <= (1e-4 if dtype == "f32" else 2e-2), w.name
 
 
 def test_static_scratch_refuses_what_does_not_fit():
