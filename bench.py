@@ -255,9 +255,10 @@ def main():
         ms_total = sum(a.elapsed_time(b) for a, b in evs)
     # per-stage durations (encode incl. merge, decode), same inputs, events on the launching stream
     wse = flare.alloc_workspace(desc, flare.OP_ENCODE)
+    wsd = flare.alloc_workspace(desc, flare.OP_DECODE)
     stage_ms = {}
     for name, fn in (("encode", lambda: flare.flare_encode(desc, Q, K, V, mask, Z, None, wse, stream)),
-                     ("decode", lambda: flare.flare_decode(desc, Q, K, Z, Y, None, stream))):
+                     ("decode", lambda: flare.flare_decode(desc, Q, K, Z, Y, None, wsd, stream))):
         pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
         for a, b in pairs:
             if flush is not None:
@@ -301,10 +302,6 @@ def main():
                    flare.flare_launch_count(desc, flare.OP_BACKWARD),
                    "note": "per GPU; forward with saved statistics, then backward"}
         del dYt, dK, dV, wsb
-    if w.dtype == "bf16" and w.M > 512:
-        # flare_decode has no workspace and runs more than 512 latents on the CUDA cores; inside flare_forward the
-        # decode runs in latent ranges on the tensor cores, so its time is the forward's less the encode's
-        stage_ms["decode"] = max(ms_total / args.steps - stage_ms["encode"], 0.0)
     clocks = sampler.stop() if rank == 0 else None
     flare.flare_check(ws)
 

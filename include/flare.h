@@ -108,11 +108,30 @@ int flare_encode(const flare_desc_t *desc, const void *Q_lat, const void *K, con
 
 /*
  * Decode (Section 3.2, decode equation; per-token sum of the design-principles appendix):
- * Y and, if lse_dec != NULL, lse_dec, from K, Q_lat and a latent sequence Z.  Needs no workspace (and therefore
- * runs more than 512 bfloat16 latents on the CUDA cores; flare_forward, which has a workspace, does not).
+ * Y and, if lse_dec != NULL, lse_dec, from K, Q_lat and a latent sequence Z.
+ * workspace: flare_workspace_bytes(desc, FLARE_OP_DECODE) bytes, or NULL.  Without a workspace the call still
+ * works, but it has nowhere to keep a flag word or partial rows: bfloat16 inputs then always take the exact form
+ * of the kernel (see flare_set_path), more than 512 bfloat16 latents run on the CUDA cores, and a bounded wait
+ * that gives up is not reported.
  */
 int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *Z, void *Y,
-                 float *lse_dec, flare_stream_t stream);
+                 float *lse_dec, void *workspace, size_t workspace_bytes, flare_stream_t stream);
+
+/*
+ * Which form of the bfloat16 tensor-core forward kernels runs (process-wide; the paper has no counterpart).
+ * Both stages are softmaxes, and a softmax is usually stabilised by subtracting the row maximum before every
+ * exponential (the exact forms: a running maximum in encode, a first pass over the scores in decode).  The fast
+ * forms skip that: float32 and bfloat16 hold 2^x for |x| < 126, so exp(score) can be formed as it stands while
+ * every |scale * q.k| stays below 96 binades (66.5 in natural units).  They check the sufficient condition
+ * |q| |k| scale log2(e) <= 96 on every key row they load, and raise a flag in the workspace header if it fails;
+ * the exact form is launched right behind and exits at once unless the flag is up, in which case it redoes the
+ * stage.  Results of the two forms agree within the forward's error bound, not bit for bit.
+ *   FLARE_PATH_AUTO   (default) fast forms for problems large enough to hide the extra launches
+ *   FLARE_PATH_EXACT  always the exact forms
+ *   FLARE_PATH_FAST   fast forms wherever the tensor-core kernels run
+ */
+enum { FLARE_PATH_AUTO = 0, FLARE_PATH_EXACT = 1, FLARE_PATH_FAST = 2 };
+int flare_set_path(int path);
 
 /*
  * The whole mixer (the paper's two-call listing in Section 3.2): encode, merge, decode on one stream.

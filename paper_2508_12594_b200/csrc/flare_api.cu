@@ -127,6 +127,22 @@ bool use_tc(const flare_desc_t *d) {
            (d->D == 16 || d->D == 32 || d->D == 64 || (d->D == 8 && d->H >= 2) || (d->D == 4 && d->H >= 4 && d->H % 2 == 0));
 }
 
+// Which form of the tensor-core forward kernels runs (flare_set_path).
+std::atomic<int> g_path{FLARE_PATH_AUTO};
+
+// The fast forms (no running maximum, see kFastMaxLog2 in flare_tc.cuh) are followed by a launch of the exact
+// form that exits at once unless it is needed: two more launches per forward, which pay off from a few tens of
+// microseconds of work.
+bool use_fast(const flare_desc_t *d) {
+    if (!use_tc(d)) return false;
+    const int path = g_path.load(std::memory_order_relaxed);
+    if (path == FLARE_PATH_EXACT) return false;
+    if (path == FLARE_PATH_FAST) return true;
+    // (measured: below 256 latents a tile has too few units for the streaming forms to beat the exact ones, which
+    // hand a whole tile's row of scores over at once)
+    return d->M >= 256 && (double)d->B * d->H * d->N * d->M >= 3.0e7;
+}
+
 // Launch plan of the tensor-core encode: `pairs` CTAs per head along the latents (two 128-latent blocks each),
 // `splits` CTAs along N, about one CTA per SM in total.
 struct TcEncodePlan {
@@ -222,10 +238,14 @@ int make_latent_map(CUtensorMap *m, const void *base, const flare_desc_t *d) {
 constexpr float kLog2e = 1.4426950408889634f;
 
 // kDz: the backward's dZ form of the kernel (V is then dY, lse_dec the decode log-sum-exp rows, pm and pl unused).
-template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false>
+// Header words of a workspace beyond the error flag: set by the fast form of encode / decode when its inputs are
+// outside the range it is valid for; the exact form that follows runs only then.
+constexpr int kRedoEncodeWord = 2, kRedoDecodeWord = 3;
+
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false>
 int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
                      const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
-                     const float *lse_dec = nullptr) {
+                     const float *lse_dec = nullptr, bool fallback = false) {
     constexpr int DG = kPair ? 2 * D : D;
     CUtensorMap tmK, tmV, tmQ;
     int rc;
@@ -235,16 +255,18 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
     const size_t smem = EncodeSmem<DG>::total();
     static std::atomic<uint64_t> smem_opt_in{0};
-    if (int rc_attr = ensure_big_smem(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody>, smem_opt_in, 227 * 1024)) return rc_attr;
+    if (int rc_attr = ensure_big_smem(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast>, smem_opt_in, 227 * 1024)) return rc_attr;
     EncodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.lse_dec = lse_dec;
     a.key_mask = mask; a.part_m = pm; a.part_l = pl; a.part_acc = pacc; a.status = status;
+    a.run_if = fallback ? status + kRedoEncodeWord : nullptr;
+    a.redo = status + kRedoEncodeWord;
     a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -343,7 +365,7 @@ int launch_bwd_token_tc(const flare_desc_t *d, int sms, const void *Q, const voi
 
 template <int D, int DRT, bool kPart, int kM>
 int launch_decode_tc_m(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
-                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart) {
+                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart, bool fallback = false) {
     CUtensorMap tmK, tmQ;
     int rc;
     if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
@@ -355,6 +377,8 @@ int launch_decode_tc_m(const flare_desc_t *d, int sms, const void *Q, const void
     DecodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.Y = (__nv_bfloat16 *)Y; a.lse_dec = lse_dec; a.status = status;
+    a.run_if = (fallback && status != nullptr) ? status + kRedoDecodeWord : nullptr;
+    a.redo = status != nullptr ? status + kRedoDecodeWord : nullptr;
     a.B = d->B; a.H = d->H; a.N = d->N; a.M = mc;
     a.mtot = d->M; a.m0 = m0; a.Ypart = Ypart;
     a.sl2 = d->scale * kLog2e;
@@ -370,18 +394,89 @@ int launch_decode_tc_m(const flare_desc_t *d, int sms, const void *Q, const void
     return FLARE_OK;
 }
 
+// The streaming (fast) form of decode: head widths 16 (and narrower) and 32, as many latents as fit shared memory.
+template <int D>
+bool decode_stream_fits(int mc) { return (D == 16 || D == 32) && DecodeStreamSmem<(D == 16 || D == 32) ? D : 16>::fits(mc); }
+
+template <int D, int DRT, bool kPart, int kM, bool kLse>
+int launch_decode_stream_l(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                           float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart) {
+    if constexpr (D == 16 || D == 32) {
+        CUtensorMap tmK, tmQ;
+        int rc;
+        if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
+        if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
+        else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
+        const size_t smem = DecodeStreamSmem<D>::total(mc);
+        static std::atomic<uint64_t> smem_opt_in{0};
+        if (int rc_attr = ensure_big_smem(decode_stream_kernel<D, DRT, kPart, kM, kLse>, smem_opt_in, 227 * 1024)) return rc_attr;
+        DecodeTcArgs a;
+        a.Q = static_cast<const __nv_bfloat16 *>(Q);
+        a.Z = Z; a.Y = (__nv_bfloat16 *)Y; a.lse_dec = lse_dec; a.status = status;
+        a.run_if = nullptr;
+        a.redo = status + kRedoDecodeWord;
+        a.B = d->B; a.H = d->H; a.N = d->N; a.M = mc;
+        a.mtot = d->M; a.m0 = m0; a.Ypart = Ypart;
+        a.sl2 = d->scale * kLog2e;
+        a.tiles = (d->N + kTile - 1) / kTile;
+        a.plan = DecodePlan{};
+        long per_head = sms / ((long)d->B * d->H);
+        const long four = (a.tiles + 3) / 4;                    // a CTA works on four tiles at a time
+        if (per_head > four) per_head = four;
+        if (per_head < 1) per_head = 1;
+        decode_stream_kernel<D, DRT, kPart, kM, kLse><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmQ, a);
+        FLARE_CUDA(cudaGetLastError());
+        return FLARE_OK;
+    } else {
+        return FLARE_ERR_UNSUPPORTED;
+    }
+}
+
+template <int D, int DRT, bool kPart, int kM>
+int launch_decode_stream_m(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                           float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart) {
+    if (lse_dec != nullptr) return launch_decode_stream_l<D, DRT, kPart, kM, true>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if constexpr (kPart) return FLARE_ERR_INVALID_ARG;          // a range of the latents always leaves its log-sum-exp
+    else return launch_decode_stream_l<D, DRT, kPart, kM, false>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+}
+
+// (the common latent counts as compile-time constants of the kernel)
+template <int D, int DRT, bool kPart>
+int launch_decode_stream(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                         float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart) {
+    if (mc == 256) return launch_decode_stream_m<D, DRT, kPart, 256>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 128) return launch_decode_stream_m<D, DRT, kPart, 128>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 64) return launch_decode_stream_m<D, DRT, kPart, 64>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    if (mc == 512) return launch_decode_stream_m<D, DRT, kPart, 512>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    return launch_decode_stream_m<D, DRT, kPart, 0>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+}
+
 // The launch's range of latents is [m0, m0 + mc) (mc = 0: all of them).  The sizes that the workloads use most have
-// forms of the kernel with the number of latents as a compile-time constant.
+// forms of the kernel with the number of latents as a compile-time constant.  fast: the form without a row maximum
+// first, then the exact form, which exits at once unless the first one found its inputs out of range (this needs
+// the flag word in a workspace header: status != null).
+template <int D, int DRT, bool kPart>
+int launch_decode_tc_f(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
+                       float *lse_dec, uint32_t *status, cudaStream_t st, int m0, int mc, float *Ypart, bool fallback) {
+    if (mc == 256) return launch_decode_tc_m<D, DRT, kPart, 256>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fallback);
+    if (mc == 128) return launch_decode_tc_m<D, DRT, kPart, 128>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fallback);
+    if (mc == 64) return launch_decode_tc_m<D, DRT, kPart, 64>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fallback);
+    if (mc == 32) return launch_decode_tc_m<D, DRT, kPart, 32>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fallback);
+    if (mc == 512) return launch_decode_tc_m<D, DRT, kPart, 512>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fallback);
+    return launch_decode_tc_m<D, DRT, kPart, 0>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fallback);
+}
+
 template <int D, int DRT = 0, bool kPart = false>
 int launch_decode_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y,
-                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0 = 0, int mc = 0, float *Ypart = nullptr) {
+                     float *lse_dec, uint32_t *status, cudaStream_t st, int m0 = 0, int mc = 0, float *Ypart = nullptr,
+                     bool fast = false) {
     if (mc == 0) mc = d->M;
-    if (mc == 256) return launch_decode_tc_m<D, DRT, kPart, 256>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
-    if (mc == 128) return launch_decode_tc_m<D, DRT, kPart, 128>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
-    if (mc == 64) return launch_decode_tc_m<D, DRT, kPart, 64>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
-    if (mc == 32) return launch_decode_tc_m<D, DRT, kPart, 32>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
-    if (mc == 512) return launch_decode_tc_m<D, DRT, kPart, 512>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
-    return launch_decode_tc_m<D, DRT, kPart, 0>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+    fast = fast && status != nullptr && decode_stream_fits<D>(mc);
+    if (fast) {
+        const int rc = launch_decode_stream<D, DRT, kPart>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart);
+        if (rc != FLARE_OK) return rc;
+    }
+    return launch_decode_tc_f<D, DRT, kPart>(d, sms, Q, K, Z, Y, lse_dec, status, st, m0, mc, Ypart, fast);
 }
 
 template <typename T>
@@ -605,6 +700,17 @@ int require_device() {
     return FLARE_OK;
 }
 
+// The fast form first (if wanted), then the exact form, which exits at once unless the fast one raised its flag.
+template <int D, bool kPair, int DRT, bool kHiLo, bool kMaskBody>
+int encode_tc_forms(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
+                    const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st, bool fast) {
+    if (fast) {
+        const int rc = launch_encode_tc<D, kPair, false, DRT, kHiLo, kMaskBody, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st);
+        if (rc != FLARE_OK) return rc;
+    }
+    return launch_encode_tc<D, kPair, false, DRT, kHiLo, kMaskBody, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st, nullptr, fast);
+}
+
 int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void *V, const uint8_t *mask, float *Z,
                 float *lse_enc, void *ws, cudaStream_t st) {
     const DeviceView di = device_info();
@@ -621,9 +727,9 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
         TcEncodePlan p = tc_encode_plan(d, di.sms);
         uint32_t *status = reinterpret_cast<uint32_t *>(base);
         // a caller that asks for lse_enc is saving Z for the backward: weights as two bf16 halves (see exp_chunk_hilo)
-#define FLARE_ENC2(DD, PAIR, DRT, MB)                                                                                     \
-    (lse_enc != nullptr ? launch_encode_tc<DD, PAIR, false, DRT, true, MB>(d, p, Q, K, V, mask, pm, pl, pacc, status, st) \
-                        : launch_encode_tc<DD, PAIR, false, DRT, false, MB>(d, p, Q, K, V, mask, pm, pl, pacc, status, st))
+        const bool fast = use_fast(d);
+#define FLARE_ENC3(DD, PAIR, DRT, MB, HL) encode_tc_forms<DD, PAIR, DRT, HL, MB>(d, p, Q, K, V, mask, pm, pl, pacc, status, st, fast)
+#define FLARE_ENC2(DD, PAIR, DRT, MB) (lse_enc != nullptr ? FLARE_ENC3(DD, PAIR, DRT, MB, true) : FLARE_ENC3(DD, PAIR, DRT, MB, false))
         // A call with a key mask has padding in every tile and takes the form that tests every element (see
         // encode_tc_kernel).  Without a mask only a last partial tile has padding and either form serves; which one
         // is faster was measured (B200): the form without the element tests where a CTA holds two latent blocks
@@ -641,6 +747,7 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
                               : FLARE_ENC(64, false, 0);
 #undef FLARE_ENC
 #undef FLARE_ENC2
+#undef FLARE_ENC3
     } else {
         SimtPlan p = simt_plan(d, di.sms);
         rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)
@@ -673,7 +780,8 @@ size_t decode_range_bytes(const flare_desc_t *d) {
 template <int D, int DRT>
 int decode_tc_any(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
                   uint32_t *status, char *range_scratch, cudaStream_t st) {
-    if (d->M <= kDecodeMaxM) return launch_decode_tc<D, DRT>(d, sms, Q, K, Z, Y, lse_dec, status, st);
+    const bool fast = use_fast(d) && status != nullptr;
+    if (d->M <= kDecodeMaxM) return launch_decode_tc<D, DRT>(d, sms, Q, K, Z, Y, lse_dec, status, st, 0, 0, nullptr, fast);
     constexpr int DR = DRT ? DRT : D;
     const int C = decode_ranges(d);
     const size_t rows = (size_t)d->B * d->N * d->H;
@@ -682,7 +790,7 @@ int decode_tc_any(const flare_desc_t *d, int sms, const void *Q, const void *K, 
     for (int c = 0; c < C; ++c) {
         const int m0 = c * kDecodeRange, mc = d->M - m0 < kDecodeRange ? d->M - m0 : kDecodeRange;
         const int rc = launch_decode_tc<D, DRT, true>(d, sms, Q, K, Z, nullptr, lpart + (size_t)c * rows, status, st, m0, mc,
-                                                Ypart + (size_t)c * rows * DR);
+                                                Ypart + (size_t)c * rows * DR, fast);
         if (rc != FLARE_OK) return rc;
     }
     decode_combine_kernel<DR><<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(Ypart, lpart, C, (long)rows,
@@ -733,11 +841,12 @@ int static_scratch_address(void **out) {
 
 // Kernels one call of `op` launches (the memset of the workspace header is not a kernel).
 int launches_for(const flare_desc_t *d, int op, int sms) {
-    const int enc = 2;                                          // encode, merge
-    const int dec = decode_in_ranges(d) ? decode_ranges(d) + 1 : 1;   // ranges of latents and their combination
+    const int f = use_fast(d) ? 2 : 1;                          // fast form, then the exact form (which may exit at once)
+    const int enc = f + 1;                                      // encode, merge
+    const int dec = decode_in_ranges(d) ? f * decode_ranges(d) + 1 : f;   // ranges of latents and their combination
     switch (op) {
         case FLARE_OP_ENCODE: return enc;
-        case FLARE_OP_DECODE: return 1;                         // without a workspace there are no ranges
+        case FLARE_OP_DECODE: return dec;                       // (given a workspace)
         case FLARE_OP_FORWARD: return enc + dec;
         case FLARE_OP_BACKWARD: {
             (void)sms;
@@ -784,7 +893,7 @@ size_t flare_workspace_bytes(const flare_desc_t *desc, int op) {
     const long rows = (long)desc->B * desc->H * desc->M;
     switch (op) {
         case FLARE_OP_ENCODE: return make_layout(partials_for(desc, device_info().sms), rows, desc->D, false).total;
-        case FLARE_OP_DECODE: return kHeaderBytes;
+        case FLARE_OP_DECODE: return kHeaderBytes + decode_range_bytes(desc);
         case FLARE_OP_FORWARD:
             return make_layout(partials_for(desc, device_info().sms), rows, desc->D, true).total + decode_range_bytes(desc);
         case FLARE_OP_BACKWARD: return bwd_layout(desc, device_info().sms).total;
@@ -826,14 +935,26 @@ int flare_encode_static_scratch(const flare_desc_t *desc, const void *Q_lat, con
 }
 
 int flare_decode(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *Z, void *Y, float *lse_dec,
-                 flare_stream_t stream) {
+                 void *workspace, size_t workspace_bytes, flare_stream_t stream) {
     int rc = check_desc(desc);
     if (rc != FLARE_OK) return rc;
     if (!Q_lat || !K || !Z || !Y) return FLARE_ERR_INVALID_ARG;
-    if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(Z) || !aligned16(Y) || (lse_dec && !aligned16(lse_dec)))
+    if (!aligned16(Q_lat) || !aligned16(K) || !aligned16(Z) || !aligned16(Y) || (lse_dec && !aligned16(lse_dec)) ||
+        (workspace && !aligned16(workspace)))
         return FLARE_ERR_INVALID_ARG;
     if ((rc = require_device()) != FLARE_OK) return rc;
-    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, nullptr, (cudaStream_t)stream);
+    if (workspace == nullptr) return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, nullptr, (cudaStream_t)stream);
+    if (workspace_bytes < flare_workspace_bytes(desc, FLARE_OP_DECODE)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    FLARE_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, (cudaStream_t)stream));
+    char *range_scratch = decode_in_ranges(desc) ? static_cast<char *>(workspace) + kHeaderBytes : nullptr;
+    return decode_impl(desc, Q_lat, K, Z, Y, lse_dec, static_cast<uint32_t *>(workspace), (cudaStream_t)stream,
+                       range_scratch);
+}
+
+int flare_set_path(int path) {
+    if (path != FLARE_PATH_AUTO && path != FLARE_PATH_EXACT && path != FLARE_PATH_FAST) return FLARE_ERR_INVALID_ARG;
+    g_path.store(path, std::memory_order_relaxed);
+    return FLARE_OK;
 }
 
 int flare_forward(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V, const uint8_t *key_mask,

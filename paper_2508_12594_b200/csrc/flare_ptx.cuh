@@ -83,6 +83,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return mbar_wait_for(bar, parity, abort_flag, code, kWaitBudgetNs);
 }
 
+// Bounded wait that polls instead of letting the hardware suspend the thread: a suspended thread resumes about
+// 150 cycles after the phase completes, a polling one within one round trip to the barrier.  For the single
+// thread whose reaction time is on the critical path of a pipeline; it takes issue slots from the warps beside it.
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t code) {
+    uint32_t spins = 0;
+    uint64_t t0 = 0;
+    while (!mbar_test(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag != 0) return false;
+            const uint64_t now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitBudgetNs) {
+                *abort_flag = code;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }

@@ -160,6 +160,106 @@ __device__ __forceinline__ void exp_chunk_hilo(const uint32_t *r, uint32_t *hi, 
     }
 }
 
+// ---------------------------------------------------------------------------- softmax without a running maximum
+// The "fast" forms of the kernels evaluate p = 2^(s * sl2) as it stands: no maximum is searched, subtracted or
+// tracked, no accumulator is ever rescaled, and the column ranges of a decode tile need no common reference.
+// float32 and bfloat16 hold 2^x for |x| < 126; with 30 binades kept free for the sums of up to 2^20 such terms times
+// values of ordinary size, that is safe while every |s * sl2| <= kFastMaxLog2.  The kernels check the sufficient
+// condition |q| |k| sl2 <= kFastMaxLog2 (Cauchy-Schwarz) on the rows they hold in shared memory and raise a flag if
+// it fails; the host then runs the exact form (running maximum) of the same kernel, which exits at once while the
+// flag is clear.
+constexpr float kFastMaxLog2 = 96.f;
+
+// Two ways to 2^x share the work.  The special-function unit (ex2.approx) delivers 16 results per clock per SM and
+// is the busiest unit of these kernels; the other half of the column pairs goes through the FMA pipe: with
+// magic = 1.5 * 2^23, t = fma(s, sl2, magic) is magic + round(x) exactly, f = fma(s, sl2, magic - t) is
+// x - round(x) in [-1/2, 1/2] with one rounding, a degree-3 polynomial gives 2^f within 7.5e-5 (the weights are
+// rounded to bfloat16, 2e-3, right after), and adding round(x) to the exponent field is one shift-and-add on the
+// bits of t.  Valid for |x| < 126, which the fast forms guarantee; scores of padded tokens (kMaskedScore) must not
+// come this way.  Measured on B200 (16 warps, scores from and weights to tensor memory): 15 results per clock per SM
+// with the special-function unit alone, 24 with every second pair on the FMA pipe.
+constexpr int kPolyDegree = 3;
+__device__ __forceinline__ float2 exp2_fma_pipe(float2 s, float2 sl2p) {
+    constexpr float kMagic = 12582912.f;                        // 1.5 * 2^23
+    const float2 magic = make_float2(kMagic, kMagic);
+    const float2 t = __ffma2_rn(s, sl2p, magic);
+    const float2 w = __ffma2_rn(t, make_float2(-1.f, -1.f), magic);   // -round(x), exact
+    const float2 f = __ffma2_rn(s, sl2p, w);
+    float2 p;
+    if (kPolyDegree == 3) {                                     // minimax on [-1/2, 1/2], relative error 7.5e-5
+        constexpr float c0 = 0.99992800f, c1 = 0.69326019f, c2 = 0.24261151f, c3 = 0.055175912f;
+        p = __ffma2_rn(make_float2(c3, c3), f, make_float2(c2, c2));
+        p = __ffma2_rn(p, f, make_float2(c1, c1));
+        p = __ffma2_rn(p, f, make_float2(c0, c0));
+    } else {                                                    // degree 2: relative error 1.7e-3
+        constexpr float c0 = 1.0004400f, c1 = 0.70345056f, c2 = 0.23845598f;
+        p = __ffma2_rn(make_float2(c2, c2), f, make_float2(c1, c1));
+        p = __ffma2_rn(p, f, make_float2(c0, c0));
+    }
+    p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
+    p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
+    return p;
+}
+
+// p = 2^(s * sl2) for NV scores, bf16 pairs to pk.  kPoly: every second pair on the FMA pipe.
+// The row sum must be that of the ROUNDED weights: without a maximum the largest weight of a row is not 1.0 but
+// some 2^x with a full mantissa, and a sum of the unrounded values would normalise it away from the rounded one
+// that multiplies the values (measured: Y off by 1.5e-2 of its RMS where one weight dominates a row, against 4e-3).
+// kSum = 0: no sum here (a ones column of the value operand lets the tensor core add the rounded weights);
+// kSum = 1: the rounded weights are widened again and added into sum2;
+// kSum = 2: as 0, and the unrounded weights are added into sum2 (for a log-sum-exp output, which must not carry the
+//           rounding of the weights: the backward rebuilds every weight from it).
+template <int NV, bool kPoly, bool kMasked, int kSum>
+__device__ __forceinline__ void exp_chunk_fast(const uint32_t *r, uint32_t *pk, float2 sl2p, float2 &sum2,
+                                               uint32_t valid = 0xffffffffu) {
+#pragma unroll
+    for (int k = 0; k < NV / 2; ++k) {
+        const float2 s = make_float2(__uint_as_float(r[2 * k]), __uint_as_float(r[2 * k + 1]));
+        float2 p;
+        if (kPoly && (k & 1)) {
+            p = exp2_fma_pipe(s, sl2p);
+        } else {
+            const float2 x = __fmul2_rn(s, sl2p);
+            p = make_float2(ptx::ex2(x.x), ptx::ex2(x.y));
+        }
+        if (kMasked) {
+            if (!((valid >> (2 * k)) & 1)) p.x = 0.f;
+            if (!((valid >> (2 * k + 1)) & 1)) p.y = 0.f;
+        }
+        pk[k] = ptx::pack_bf16(p.x, p.y);
+        if (kSum == 1) sum2 = __fadd2_rn(sum2, make_float2(__uint_as_float(pk[k] << 16), __uint_as_float(pk[k] & 0xffff0000u)));
+        if (kSum == 2) sum2 = __fadd2_rn(sum2, p);
+    }
+}
+
+// Largest squared norm among the rows [lane, lane + 32, ...) < rows of a [rows, RB / 2] bf16 tile in shared memory
+// (the 16-byte chunks of a row are permuted by the swizzle, which a sum over the whole row does not see).
+template <int RB>
+__device__ __forceinline__ float tile_max_norm2(const uint8_t *tile, int rows, int lane) {
+    float best = 0.f;
+    for (int r = lane; r < rows; r += 32) {
+        float n2 = 0.f;
+#pragma unroll
+        for (int c = 0; c < RB / 16; ++c) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(tile + (size_t)r * RB + c * 16);
+            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float a = __uint_as_float(u[k] << 16), b = __uint_as_float(u[k] & 0xffff0000u);
+                n2 = fmaf(a, a, fmaf(b, b, n2));
+            }
+        }
+        if (!(n2 <= 3.0e38f)) n2 = INFINITY;                    // a row with a NaN or an infinity fails every check
+        best = fmaxf(best, n2);
+    }
+    return best;
+}
+__device__ __forceinline__ float warp_max_nan(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
 // ------------------------------------------------------------------------------------------------ decode
 // How the four softmax groups share tensor memory in decode.  `cs` groups split the M score columns of one
 // buffer into ranges of `part_w` columns (the last may be shorter); `nbuf` buffers of `cb` columns hold
@@ -235,6 +335,8 @@ struct DecodeTcArgs {
     __nv_bfloat16 *Y;    // [B,N,H,D]
     float *lse_dec;      // [B,N,H] or null
     uint32_t *status;    // workspace header or null
+    const uint32_t *run_if;   // exact forms: null, or a word that must be non-zero for the kernel to do anything
+    uint32_t *redo;           // fast forms: set to 1 if a score may lie outside the range they are valid for
     int B, H, N, M;      // M: latents this launch works on (all of them, or a range of at most 512)
     int mtot, m0;        // latents per head in Q and Z, and the first one of this launch's range
     float *Ypart;        // kPart form of the kernel: [B,N,H,D] float32, rows normalised over the range go here instead
@@ -279,6 +381,7 @@ struct DecodeSmem {
 template <int D, int DRT = 0, bool kPart = false, int kM = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
+    if (a.run_if != nullptr && *a.run_if == 0) return;          // behind the streaming form, as a fallback that was not needed
     constexpr bool kHalf = DRT != 0;
     constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     using G = TileGeom<D>;
@@ -390,6 +493,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int r = 0; r < M; r += 16)
                     ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * a.mtot + a.m0 + r);
             }
+        }
+        if (lane == 0) {
             for (int i = 0; i < ntiles; ++i) {
                 const int s = i % nstages;
                 if (!ptx::mbar_wait(bar(K_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrDecode | 1)) break;
@@ -604,6 +709,414 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
 }
 
+// ------------------------------------------------------------------------------------- decode, streaming form
+// Decode without a row maximum (see kFastMaxLog2) needs no whole row of scores before the first exponential, so
+// it can run as a stream like encode: a group owns a whole token tile (tokens on the 128 lanes; the four groups of
+// a CTA work on four different tiles) and walks the latents in units of 32 columns on two alternating score
+// buffers:  S_unit = K_tile Q_unit^T,  P = 2^(S sl2) as packed bf16 back over the scores,
+// Y += P [Z_hi | Z_lo | 1]_unit.  Units follow one another across tile boundaries without a pause: the rows of a
+// finished tile are normalised and stored after the first unit of the next one.  The accumulator column after
+// [P Z_hi | P Z_lo] is the row's sum of rounded weights (see exp_chunk_fast).  D = 32: Z_lo enters as a second,
+// accumulating MMA into the columns of Z_hi, which keeps the accumulator at 48 columns.
+//
+// What shapes the pipeline (measured on B200): the thread that issues a tcgen05.mma or a tcgen05.commit is held
+// about 130 cycles per instruction, a barrier flips 170 cycles after its commit was issued, and a waiting warp
+// notices 100 to 200 cycles later.  A group's issuing thread is therefore its bottleneck as soon as it has more
+// than a handful of such instructions per unit (with separate commits and waits for scores and weights: 1300
+// cycles per unit, measured with the arithmetic taken out).  Its loop is: wait for the weights of unit n; the
+// two value MMAs of unit n; the score MMA of unit n + 2 into the buffer those weights have just been read from
+// (the tensor core runs a thread's MMAs in order); ONE commit, which tells the threads both that the scores of
+// unit n + 2 are there and that everything before them is done.
+template <int D>
+struct DecodeStreamSmem {
+    using G = TileGeom<D>;
+    static constexpr size_t kBarBytes = 1024;
+    __host__ __device__ static int stages(int M) {
+        int s = 8;
+        while (s > 4 && (size_t)s * G::TILE_BYTES + (size_t)4 * M * G::RB + kBarBytes + 2048 > 227 * 1024) --s;
+        return s;
+    }
+    __host__ __device__ static size_t q_off(int M) { return (size_t)stages(M) * G::TILE_BYTES; }
+    __host__ __device__ static size_t z_off(int M) { return q_off(M) + (size_t)M * G::RB; }      // [hi | lo | ones], M rows each
+    __host__ __device__ static size_t bar_off(int M) { return align_up(z_off(M) + (size_t)3 * M * G::RB, 1024); }
+    __host__ __device__ static size_t total(int M) {
+        size_t t = bar_off(M) + kBarBytes + 1024;
+        return t < kTcMinSmem ? kTcMinSmem : t;
+    }
+    __host__ __device__ static bool fits(int M) { return bar_off(M) + kBarBytes + 1024 <= 227 * 1024; }
+};
+
+// kM: 0, or the number of latents of the launch as a compile-time constant (a multiple of 64): the unit loops are
+// then unrolled and every descriptor offset, buffer index and barrier parity within a tile is a constant, which
+// matters most for the issuing thread (its scalar instructions wait for issue slots among the softmax warps).
+// kLse: the log-sum-exp rows are wanted (lse_dec; always with kPart): the threads then also add up the unrounded weights.
+template <int D, int DRT = 0, bool kPart = false, int kM = 0, bool kLse = false>
+__global__ void __launch_bounds__(kTcThreads, 1)
+decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
+    static_assert(D == 16 || D == 32, "head widths 16 (and narrower, as part of 16) and 32");
+    constexpr bool kHalf = DRT != 0;
+    constexpr int DR = kHalf ? DRT : D;                         // head width in memory
+    using G = TileGeom<D>;
+    using SM = DecodeStreamSmem<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    static_assert(kM % 64 == 0, "compile-time latent counts are multiples of 64");
+    const int M = kM ? kM : a.M;
+    const int nstages = SM::stages(M);
+    uint8_t *sK = smem;
+    uint8_t *sQ = smem + SM::q_off(M);
+    uint8_t *sZ = smem + SM::z_off(M);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off(M));
+    constexpr int NG = kSoftmaxGroups, kMaxStages = 8, UNIT = 32;
+    // S_FULL[2] per group: the scores of a unit are in its buffer (and all earlier MMAs of the group are done);
+    // P_FULL[2]: the unit's weights are over them (one arrival per warp); Y_FULL / Y_FREE: a tile's rows are complete / read
+    enum { K_FULL = 0, K_EMPTY = K_FULL + kMaxStages, Q_FULL = K_EMPTY + kMaxStages, S_FULL = Q_FULL + 1,
+           P_FULL = S_FULL + 2 * NG, Y_FULL = P_FULL + 2 * NG, Y_FREE = Y_FULL + NG, NBARS = Y_FREE + NG };
+    static_assert(NBARS * 8 + 16 <= SM::kBarBytes, "barrier area too small");
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    constexpr int Y_COL = 2 * UNIT, GROUP_COLS = 128;          // a group's columns: two score buffers, then 48 of Y
+    constexpr int YN = 48;                                      // N of the value MMA that carries the ones block
+    constexpr int SUM_COL = 32;                                 // accumulator column of the row sum
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int off = kHalf ? narrow_offset(h, DR) : 0;
+    const int t_begin = (int)((long)a.tiles * blockIdx.x / gridDim.x);
+    const int t_end = (int)((long)a.tiles * (blockIdx.x + 1) / gridDim.x);
+    const int ntiles = t_end - t_begin;
+    const int units = (M + UNIT - 1) / UNIT;                    // per tile; the last may have 16 columns
+    auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NBARS; ++i) {
+            const bool by_warps = (i >= P_FULL && i < P_FULL + 2 * NG) || (i >= Y_FREE && i < Y_FREE + NG);
+            ptx::mbar_init(bar(i), by_warps ? 4u : 1u);
+        }
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmK);
+        ptx::prefetch_tensormap(&tmQ);
+    }
+    if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+    {   // Z_bh -> [hi | lo | ones] blocks of M latent-major rows in the swizzled layout of an MN-major B operand
+        const float *Zg = a.Z + (((size_t)b * a.H + h) * a.mtot + a.m0) * DR;
+        if (kHalf) {
+            for (int i = threadIdx.x; i < M * (D / 8); i += kTcThreads) {
+                reinterpret_cast<uint4 *>(sQ)[i] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4 *>(sZ)[i] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4 *>(sZ + (size_t)M * G::RB)[i] = make_uint4(0, 0, 0, 0);
+            }
+            __syncthreads();
+            if constexpr (DR == 4) {
+                stage_rows4<D>(sQ, a.Q + ((size_t)h * a.mtot + a.m0) * DR, M, off);
+                stage_rows4_hilo<D>(sZ, sZ + (size_t)M * G::RB, Zg, M, off);
+            } else {
+                for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+                    const int m = i / (DR / 8), c = i % (DR / 8);
+                    *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) =
+                        *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * a.mtot + a.m0 + m) * DR + c * 8);
+                }
+            }
+        }
+        constexpr int ZC = DR >= 8 ? DR / 8 : 1;
+        for (int i = threadIdx.x; i < (DR >= 8 ? M * ZC : 0); i += kTcThreads) {
+            const int m = i / ZC, c = i % ZC;
+            const float4 lo = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8);
+            const float4 hi = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8 + 4);
+            const float z[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            uint32_t vh[4], vl[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                vh[k] = ptx::pack_bf16(z[2 * k], z[2 * k + 1]);
+                vl[k] = ptx::pack_bf16(z[2 * k] - __uint_as_float(vh[k] << 16), z[2 * k + 1] - __uint_as_float(vh[k] & 0xffff0000u));
+            }
+            uint8_t *dst = sZ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4);
+            *reinterpret_cast<uint4 *>(dst) = make_uint4(vh[0], vh[1], vh[2], vh[3]);
+            *reinterpret_cast<uint4 *>(dst + (size_t)M * G::RB) = make_uint4(vl[0], vl[1], vl[2], vl[3]);
+        }
+        uint8_t *ones = sZ + (size_t)2 * M * G::RB;             // a one in column 0 of every latent row
+        for (int i = threadIdx.x; i < M * (G::RB / 16); i += kTcThreads) {
+            const int m = i / (G::RB / 16), c = i % (G::RB / 16);
+            *reinterpret_cast<uint4 *>(ones + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) = make_uint4(c == 0 ? 0x00003F80u : 0u, 0, 0, 0);
+        }
+        ptx::fence_proxy_async_smem();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tm = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            if (kHalf) {
+                ptx::mbar_arrive(bar(Q_FULL));
+            } else {
+                ptx::mbar_arrive_expect_tx(bar(Q_FULL), (uint32_t)(M * G::RB));
+                for (int r = 0; r < M; r += 16)
+                    ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * a.mtot + a.m0 + r);
+            }
+        }
+        // The whole warp walks the tiles: lane 0 issues the loads; all lanes check the key rows of the tile a stage held
+        // before it is overwritten: |q| |k| sl2 <= kFastMaxLog2 for every latent row of the launch (whole rows: in
+        // the narrow forms they hold the neighbouring heads' features too, which only makes the check stricter).
+        bool tame = warp_wait(bar(Q_FULL), 0, abort_flag, kErrDecode | 9);
+        const float q2 = warp_max_nan(tile_max_norm2<G::RB>(sQ, M, lane));
+        const float lim = kFastMaxLog2 / a.sl2;
+        const float k2_limit = lim * lim / fmaxf(q2, 1e-30f);
+        if (!(q2 <= 3.0e38f)) tame = false;
+        auto check_tile = [&](int j) {
+            const int sj = j % nstages;
+            if (!warp_wait(bar(K_FULL + sj), (j / nstages) & 1, abort_flag, kErrDecode | 10)) return;
+            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sK + (size_t)sj * G::TILE_BYTES, kTile, lane));
+            if (!(k2 <= k2_limit)) tame = false;
+        };
+        for (int i = 0; i < ntiles; ++i) {
+            const int s = i % nstages;
+            if (i >= nstages) check_tile(i - nstages);
+            if (!warp_wait(bar(K_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrDecode | 1)) break;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(bar(K_FULL + s), G::TILE_BYTES);
+                ptx::tma_load_3d(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), &tmK, bar(K_FULL + s), h * DR - off,
+                                 (t_begin + i) * kTile, b);
+            }
+        }
+        for (int j = ntiles > nstages ? ntiles - nstages : 0; j < ntiles; ++j) check_tile(j);
+        if (!tame && lane == 0 && a.redo != nullptr) *a.redo = 1u;
+    } else if (warp < kFirstSoftmaxWarp) {
+        const int g = warp - kFirstIssuerWarp;
+        const int mytiles = (ntiles - g + NG - 1) / NG;          // tiles g, g + 4, ... of the CTA's range
+        if (lane == 0 && mytiles > 0) {
+            const uint32_t gcol = tm + g * GROUP_COLS;
+            const uint32_t idescY = ptx::instr_desc_bf16(128, YN, 0, 1);
+            const uint32_t idescLo = ptx::instr_desc_bf16(128, D, 0, 1);       // D = 32: the accumulating Z_lo product
+            const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ);
+            // value operand: Z_hi rows of the unit; next block along N: Z_lo (D = 16, then the ones block) or the ones
+            // block (D = 32), LBO bytes further on
+            const uint64_t zdesc = ptx::smem_desc(ptx::smem_u32(sZ), (uint32_t)((D == 16 ? 1 : 2) * M * G::RB), G::SBO, G::SWZ);
+            const uint64_t zlo = ptx::smem_desc(ptx::smem_u32(sZ + (size_t)M * G::RB), (uint32_t)G::SBO, G::SBO, G::SWZ);
+            const int total = mytiles * units;
+            bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrDecode | 2);
+            const uint32_t kstep = (uint32_t)(G::TILE_BYTES >> 4);
+            const uint64_t kdesc0 = ptx::smem_desc(ptx::smem_u32(sK), 16, G::SBO, G::SWZ);
+            if constexpr (kM != 0) {
+                // Unrolled over the tile's units: unit c of every tile uses buffer c & 1 (the number of units is even),
+                // so within a tile every buffer, descriptor offset and barrier parity is a constant.
+                constexpr int U = kM / UNIT;
+                constexpr uint32_t idescS = ptx::instr_desc_bf16(128, UNIT, 0, 0);
+                const uint32_t sfull = bar(S_FULL + 2 * g), pfull = bar(P_FULL + 2 * g);
+                int stage = g % nstages, wrap = 0;               // K stage of the tile whose scores are issued next, and its phase
+                uint64_t kdesc = 0;
+                auto scores = [&](int c) {                        // S of unit c (a constant after unrolling) of the tile at kdesc, and the commit
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k)
+                        ptx::mma_ss(gcol + (c & 1) * UNIT, kdesc + 2 * k, qdesc + (uint64_t)((c * UNIT * G::RB) >> 4) + 2 * k, idescS, k > 0);
+                    ptx::mma_commit(sfull + 8 * (c & 1));
+                };
+                auto open_tile = [&]() -> bool {                  // wait for the K tile of the S stream's next tile
+                    if (!ptx::mbar_wait(bar(K_FULL + stage), (uint32_t)wrap, abort_flag, kErrDecode | 3)) return false;
+                    ptx::tc_fence_after();
+                    kdesc = kdesc0 + (uint64_t)(kstep * (uint32_t)stage);
+                    return true;
+                };
+                auto close_tile = [&]() {                         // its last scores are issued: the stage is free, on to the next tile
+                    ptx::mma_commit(bar(K_EMPTY + stage));
+                    stage += NG;
+                    if (stage >= nstages) { stage -= nstages; wrap ^= 1; }
+                };
+                ok = ok && open_tile();
+                if (ok) {
+                    scores(0);
+                    scores(1);
+                    if (U == 2) close_tile();
+                }
+                for (int tu = 0; ok && tu < mytiles; ++tu) {
+                    const uint32_t par = (uint32_t)((tu * (U / 2)) & 1);    // parity of the tile's first two units on their buffers
+                    const bool more = tu + 1 < mytiles;
+#pragma unroll
+                    for (int c = 0; c < U; ++c) {
+                        if (!ptx::mbar_spin(pfull + 8 * (c & 1), par ^ (uint32_t)((c >> 1) & 1), abort_flag, kErrDecode | 5)) { ok = false; break; }
+                        if (c == 0 && tu > 0 && !ptx::mbar_spin(bar(Y_FREE + g), (uint32_t)((tu - 1) & 1), abort_flag, kErrDecode | 11)) { ok = false; break; }
+                        ptx::tc_fence_after();
+                        const uint32_t pcol = gcol + (c & 1) * UNIT;
+                        const uint64_t zr = zdesc + (uint64_t)((c * UNIT * G::RB) >> 4), zl = zlo + (uint64_t)((c * UNIT * G::RB) >> 4);
+                        ptx::mma_ts(gcol + Y_COL, pcol, zr, idescY, c == 0 ? 0u : 1u);
+                        if (D == 32) ptx::mma_ts(gcol + Y_COL, pcol, zl, idescLo, 1u);
+                        ptx::mma_ts(gcol + Y_COL, pcol + 8, zr + (uint64_t)(G::RB), idescY, 1u);
+                        if (D == 32) ptx::mma_ts(gcol + Y_COL, pcol + 8, zl + (uint64_t)(G::RB), idescLo, 1u);
+                        if (c == U - 1) ptx::mma_commit(bar(Y_FULL + g));
+                        // the scores of the unit two further on go into the buffer just read; the commit behind them covers
+                        // the value MMAs above as well
+                        if (c + 2 < U) {
+                            scores(c + 2);
+                            if (c + 2 == U - 1) close_tile();
+                        } else if (more) {
+                            if (c + 2 == U && !open_tile()) { ok = false; break; }
+                            scores(c + 2 - U);
+                            if (c + 2 - U == U - 1) close_tile();
+                        }
+                    }
+                }
+            } else {
+                // This thread's own instructions are on the critical path of the group (they run one at a time, each
+                // waiting for its issue slot among the softmax warps), so both streams of work below keep their
+                // position in running counters instead of dividing: the score units (two ahead of the value units) ...
+                int s_c = 0, s_stage = g % nstages, s_wrap = (g / nstages) & 1, s_n = 0;   // chunk, K stage and its phase, unit
+                const int last_nn = M - (units - 1) * UNIT;
+                const uint32_t idescS_full = ptx::instr_desc_bf16(128, UNIT, 0, 0), idescS_last = ptx::instr_desc_bf16(128, last_nn, 0, 0);
+                auto issue_scores = [&]() -> bool {                   // (the caller commits)
+                    if (s_c == 0) {
+                        if (!ptx::mbar_wait(bar(K_FULL + s_stage), (uint32_t)s_wrap, abort_flag, kErrDecode | 3)) return false;
+                        ptx::tc_fence_after();
+                    }
+                    const uint64_t kdesc = kdesc0 + (uint64_t)(kstep * (uint32_t)s_stage);
+                    const uint64_t qd = qdesc + (uint64_t)((uint32_t)(s_c * UNIT * G::RB) >> 4);
+                    const uint32_t idescS = s_c == units - 1 ? idescS_last : idescS_full;
+                    const uint32_t w = (uint32_t)(s_n & 1);
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gcol + w * UNIT, kdesc + 2 * k, qd + 2 * k, idescS, k > 0);
+                    ptx::mma_commit(bar(S_FULL + 2 * g) + 8 * w);
+                    ++s_n;
+                    if (++s_c == units) {                           // the tile's last scores: its stage is free, on to the next tile
+                        ptx::mma_commit(bar(K_EMPTY + s_stage));
+                        s_c = 0;
+                        s_stage += NG;
+                        if (s_stage >= nstages) { s_stage -= nstages; s_wrap ^= 1; }
+                    }
+                    return true;
+                };
+                for (int n = 0; ok && n < 2 && n < total; ++n) ok = issue_scores();
+                // ... and the value units
+                int c = 0, tu = 0;
+                for (int n = 0; ok && n < total; ++n) {
+                    const uint32_t w = (uint32_t)(n & 1);           // the unit's buffer: its weights lie over its scores
+                    if (!ptx::mbar_spin(bar(P_FULL + 2 * g) + 8 * w, (uint32_t)((n >> 1) & 1), abort_flag, kErrDecode | 5)) break;
+                    // a tile's first value MMA overwrites the accumulator: the previous tile's rows must have been read
+                    if (c == 0 && tu > 0 && !ptx::mbar_spin(bar(Y_FREE + g), (uint32_t)((tu - 1) & 1), abort_flag, kErrDecode | 11)) break;
+                    ptx::tc_fence_after();
+                    const int subs = (c == units - 1 ? last_nn : UNIT) / 16;
+                    const uint64_t rowoff = (uint64_t)((uint32_t)(c * UNIT * G::RB) >> 4);
+                    const uint32_t pcol = gcol + w * UNIT;
+                    ptx::mma_ts(gcol + Y_COL, pcol, zdesc + rowoff, idescY, c == 0 ? 0u : 1u);
+                    if (D == 32) ptx::mma_ts(gcol + Y_COL, pcol, zlo + rowoff, idescLo, 1u);
+                    if (subs == 2) {                                // the unit's second 16 latents: 8 packed columns, 16 rows of Z on
+                        ptx::mma_ts(gcol + Y_COL, pcol + 8, zdesc + rowoff + (uint64_t)(G::RB), idescY, 1u);
+                        if (D == 32) ptx::mma_ts(gcol + Y_COL, pcol + 8, zlo + rowoff + (uint64_t)(G::RB), idescLo, 1u);
+                    }
+                    if (++c == units) {
+                        ptx::mma_commit(bar(Y_FULL + g));
+                        c = 0;
+                        ++tu;
+                    }
+                    if (n + 2 < total && !(ok = issue_scores())) break;   // into the buffer just read; its commit covers the value MMAs too
+                }
+            }
+        }
+    } else {
+        const int g = (warp - kFirstSoftmaxWarp) >> 2;
+        const int mytiles = (ntiles - g + NG - 1) / NG;
+        const int row = ((warp & 3) << 5) + lane;               // TMEM lane = token within the tile
+        const uint32_t gcol = tm + ((uint32_t)((warp & 3) << 5) << 16) + g * GROUP_COLS;
+        const float2 sl2p = make_float2(a.sl2, a.sl2);
+        float2 sum2 = make_float2(0.f, 0.f);                    // kLse: the tile's row sum of unrounded weights so far
+        float l_exact = 0.f;                                    // ... and that of the tile whose rows are still to be written
+        constexpr int kSum = kLse ? 2 : 0;
+        // normalise and store the rows of tile tu (this group's tu-th), whose value MMAs are all issued
+        auto epilogue = [&](int tu) -> bool {
+            if (!warp_wait(bar(Y_FULL + g), tu & 1, abort_flag, kErrDecode | 7)) return false;
+            ptx::tc_fence_after();
+            uint32_t y[48];
+            ptx::tmem_ld32(gcol + Y_COL, *reinterpret_cast<uint32_t(*)[32]>(y));
+            ptx::tmem_ld16(gcol + Y_COL + 32, y + 32);
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(Y_FREE + g));    // the accumulator may be overwritten
+            const float l = __uint_as_float(y[SUM_COL]);
+            const float inv = 1.f / l;
+            const int n = (t_begin + g + tu * NG) * kTile + row;
+            if (n < a.N) {
+                // the head's DR values: accumulator columns [off, off + DR) (off is 0 except for every other head of width 4)
+                float v[DR];
+#pragma unroll
+                for (int k = 0; k < DR; ++k) {
+                    if (D == 16) {
+                        const float a0 = __uint_as_float(y[k]) + __uint_as_float(y[16 + k]);
+                        const float a4 = DR == 4 ? __uint_as_float(y[4 + k]) + __uint_as_float(y[20 + k]) : a0;
+                        v[k] = ((DR == 4 && off) ? a4 : a0) * inv;
+                    } else {
+                        v[k] = __uint_as_float(y[k]) * inv;
+                    }
+                }
+                const size_t rowidx = ((size_t)b * a.N + n) * a.H + h;
+                if (kPart) {
+                    float4 *pd = reinterpret_cast<float4 *>(a.Ypart + rowidx * DR);
+#pragma unroll
+                    for (int k = 0; k < DR / 4; ++k) pd[k] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+                } else if (DR == 4) {
+                    *reinterpret_cast<uint2 *>(a.Y + rowidx * DR) = make_uint2(ptx::pack_bf16(v[0], v[1]), ptx::pack_bf16(v[2], v[3]));
+                } else {
+                    uint4 *dst = reinterpret_cast<uint4 *>(a.Y + rowidx * DR);
+#pragma unroll
+                    for (int k = 0; k < DR / 8; ++k)
+                        dst[k] = make_uint4(ptx::pack_bf16(v[8 * k], v[8 * k + 1]), ptx::pack_bf16(v[8 * k + 2], v[8 * k + 3]),
+                                            ptx::pack_bf16(v[8 * k + 4], v[8 * k + 5]), ptx::pack_bf16(v[8 * k + 6], v[8 * k + 7]));
+                }
+                if (kLse) a.lse_dec[rowidx] = log2f(l_exact) * 0.6931471805599453f;
+            }
+            return true;
+        };
+        bool ok = true;
+        int n = 0;                                              // unit counter of this group's stream
+        const int total = mytiles * units;
+        // A wait on a barrier costs a warp about 150 cycles even when the phase is long complete, and the warp has
+        // nothing else to do meanwhile.  So the wait for the next unit's scores is asked early, without blocking,
+        // before the exponentials of this unit, and falls back to a blocking wait only if the answer was no.
+        bool s_ready = false;
+        for (int tu = 0; ok && tu < mytiles; ++tu) {
+            for (int c = 0; ok && c < units; ++c, ++n) {
+                const int w = n & 1;
+                const int nn = kM ? UNIT : (M - c * UNIT < UNIT ? M - c * UNIT : UNIT);
+                if (!s_ready && !(ok = warp_wait(bar(S_FULL + 2 * g + w), (n >> 1) & 1, abort_flag, kErrDecode | 6))) break;
+                ptx::tc_fence_after();
+                uint32_t r[32], pk[16];
+                if (nn == UNIT) ptx::tmem_ld32(gcol + w * UNIT, r);
+                else ptx::tmem_ld16(gcol + w * UNIT, r);
+                ptx::tmem_wait_ld();
+                bool s_probe = false;
+                if (nn == UNIT) {
+                    exp_chunk_fast<16, true, false, kSum>(r, pk, sl2p, sum2);
+                    s_probe = n + 1 < total && ptx::mbar_test(bar(S_FULL + 2 * g + (w ^ 1)), ((n + 1) >> 1) & 1);
+                    exp_chunk_fast<16, true, false, kSum>(r + 16, pk + 8, sl2p, sum2);
+                    ptx::tmem_st16(gcol + w * UNIT, pk);
+                } else {
+                    exp_chunk_fast<16, true, false, kSum>(r, pk, sl2p, sum2);
+                    ptx::tmem_st8(gcol + w * UNIT, pk);
+                }
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar(P_FULL + 2 * g + w));
+                s_ready = __all_sync(0xffffffffu, s_probe);
+                // the previous tile's rows, while the tensor core works on this unit
+                if (c == 0 && tu > 0) ok = epilogue(tu - 1);
+                if (kLse && c == units - 1) {                   // the tile's sum is complete; the next tile starts its own
+                    l_exact = sum2.x + sum2.y;
+                    sum2 = make_float2(0.f, 0.f);
+                }
+            }
+        }
+        if (ok && mytiles > 0) epilogue(mytiles - 1);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == kFirstIssuerWarp) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tm, 512);
+    }
+    if (threadIdx.x == 0 && *abort_flag != 0 && a.status != nullptr) atomicCAS(a.status, 0u, *abort_flag);
+}
+
 // Decode over more latents than one launch holds: every launch decodes a range of the latents into float32 rows
 // normalised over that range (Ypart[c]) with the range's log-sum-exp (lse_part[c]); this kernel joins the C ranges,
 //   lse = log sum_c exp(lse_c),   Y = sum_c exp(lse_c - lse) Ypart[c],
@@ -658,6 +1171,8 @@ struct EncodeTcArgs {
     const uint8_t *key_mask;  // [B,N] or null
     float *part_m, *part_l, *part_acc;
     uint32_t *status;
+    const uint32_t *run_if;   // exact forms: null, or a word that must be non-zero for the kernel to do anything
+    uint32_t *redo;           // fast forms: set to 1 if a score may lie outside the range they are valid for
     int B, H, N, M;
     float scale, sl2;
     int tiles;        // ceil(N / 128)
@@ -678,8 +1193,10 @@ struct EncodeSmem {
     // score bias of padded tokens: per stage a [128 tokens, 16] bf16 tile, then one [128 latents, 16] tile of ones
     static constexpr size_t kBiasTile = kTile * 32;
     __host__ __device__ static size_t bias_off() { return (col_off() + kColBytes + 1023) & ~(size_t)1023; }
+    // fast form: a [128 tokens, DG] tile with a one in column 0 of every row, the value operand's second block along N
+    __host__ __device__ static size_t ones_off() { return (bias_off() + (kEncStages + 1) * kBiasTile + 1023) & ~(size_t)1023; }
     __host__ __device__ static size_t total() {
-        size_t t = bias_off() + (kEncStages + 1) * kBiasTile + 1024;
+        size_t t = ones_off() + (size_t)kTile * G::RB + 1024;
         return t < kTcMinSmem ? kTcMinSmem : t;
     }
 };
@@ -721,10 +1238,16 @@ constexpr float kDeadBelow = -1.0e29f;
 // kMaskBody: padded tokens are handled by a second form of the unit body that tests every element (the form for
 // calls with a key mask, where every tile has padding); without it they are handled in the scores (kMaskedScore),
 // which costs a bias tile and one more MMA per unit of the tiles that have padding, and nothing elsewhere.
-template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false>
+//
+// kFast: no running maximum (see kFastMaxLog2): weights 2^(s * sl2) as they stand, half of them by the polynomial
+// on the FMA pipe (not with kHiLo, whose point is accuracy), no rescaling, partial maximum 0.  The producer warp
+// checks the norms of the key rows of every tile it has loaded against those of the CTA's latent rows.
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
+    static_assert(!(kFast && kDz), "the dZ form has no maximum to drop");
+    if (!kFast && a.run_if != nullptr && *a.run_if == 0) return;      // the exact form as a fallback that was not needed
     constexpr bool kHalf = DRT != 0;
     static_assert(!(kPair && kHalf), "head pairing and the narrow form exclude each other");
     constexpr int DG = kPair ? 2 * D : D;
@@ -740,6 +1263,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // per group: S_FULL and P_FULL for each of its two score buffers, PV_DONE (one phase per unit), ACC_DONE
     enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_FULL = S_FULL + 2 * NG,
            PV_DONE = P_FULL + 2 * NG, ACC_DONE = PV_DONE + NG, Q_FULL = ACC_DONE + NG, NBARS };
+    static_assert(NBARS * 8 + 8 <= 512, "barrier area too small");
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -763,6 +1287,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     constexpr int HALF = kTile / 2;
     constexpr int UNIT = 32;         // tokens per unit of work of a group
     constexpr uint32_t NCOLS = 512;
+    // Fast form with single weights: the value operand gets a second block along N whose column 0 is all ones, so
+    // accumulator column DG is the sum of the rounded weights (see exp_chunk_fast); where the accumulator has no
+    // room for it (DG = 64) the threads add the rounded weights themselves.
+    constexpr bool kOnes = kFast && !kHiLo && DG + 16 <= 2 * UNIT;
+    constexpr int kSumMode = kOnes ? 0 : 1;
+    uint8_t *sOnes = smem + SM::ones_off();
+    constexpr int ACC_COL = 2 * UNIT;                           // a group's columns: two score buffers, then the accumulator
 
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
 
@@ -770,7 +1301,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // a K/V tile is released by the issuers of all the groups that use it
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
-            ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? 128u
+            ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? (kFast ? 4u : 128u)   // fast form: one arrival per warp
                                    : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users
                                    : (i >= KV_FULL && i < KV_FULL + kEncStages) ? 2u : 1u);   // the TMA loads, the bias tile
         *abort_flag = 0;
@@ -790,6 +1321,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int r = threadIdx.x; r < kTile; r += kTcThreads) {   // row r = [1, 0, ..., 0]: the first 16-byte chunk, swizzled
             reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r)] = make_uint4(0x00003F80u, 0, 0, 0);
             reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r) ^ 1] = make_uint4(0, 0, 0, 0);
+        }
+    }
+    if (kOnes) {
+        for (int i = threadIdx.x; i < kTile * (G::RB / 16); i += kTcThreads) {
+            const int r = i / (G::RB / 16), ch = i % (G::RB / 16);
+            *reinterpret_cast<uint4 *>(sOnes + (size_t)r * G::RB + ((ch ^ G::swz(r)) << 4)) =
+                make_uint4(ch == 0 ? 0x00003F80u : 0u, 0, 0, 0);
         }
     }
     if (kPair) {
@@ -831,10 +1369,29 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
             }
         }
+        // Fast form: the largest |k|^2 a tile may hold so that |q| |k| sl2 <= kFastMaxLog2 for the CTA's latent rows.
+        // (Whole rows of both operands: in the head-pair and narrow forms they hold the neighbouring heads' features
+        // too, which only makes the check stricter.)
+        float k2_limit = 0.f;
+        bool tame = true;
+        if (kFast) {
+            tame = warp_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 8);
+            const float q2 = warp_max_nan(tile_max_norm2<G::RB>(sQ, 2 * kTile, lane));
+            const float lim = kFastMaxLog2 / a.sl2;
+            k2_limit = lim * lim / fmaxf(q2, 1e-30f);
+            if (!(q2 <= 3.0e38f)) tame = false;                 // NaN or infinity in Q
+        }
+        auto check_tile = [&](int j) {                           // K tile j (relative to t_begin), still in its stage
+            const int sj = j % kEncStages;
+            if (!warp_wait(bar(KV_FULL + sj), (j / kEncStages) & 1, abort_flag, kErrEncode | 9)) return;
+            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sKV + (size_t)sj * 2 * G::TILE_BYTES, kTile, lane));
+            if (!(k2 <= k2_limit)) tame = false;
+        };
         // The whole warp walks the tiles: lane 0 waits for the stage and issues the loads; for a tile with padding
         // (masked tokens, or tokens beyond N) every lane first writes four rows of the stage's bias tile.
         for (int i = 0; i < nt; ++i) {
             const int s = i % kEncStages, t = t_begin + i;
+            if (kFast && i >= kEncStages) check_tile(i - kEncStages);   // the tile this stage held, before it is overwritten
             if (!warp_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
             const bool plain = kDz || kMaskBody || (a.key_mask == nullptr && (t + 1) * kTile <= a.N);
             if (!plain) {
@@ -859,17 +1416,21 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR - off, t * kTile, b);
             }
         }
+        if (kFast) {
+            for (int j = nt > kEncStages ? nt - kEncStages : 0; j < nt; ++j) check_tile(j);   // the tiles still in their stages
+            if (!tame && lane == 0) *a.redo = 1u;
+        }
     } else if (warp < kFirstSoftmaxWarp) {
         const int g = warp - kFirstIssuerWarp;                  // the group this warp issues MMAs for
         const int j = g >> 1, c = g & 1;                        // its slot and column half
         if (lane == 0 && j < nslots) {
             const uint32_t idescS = ptx::instr_desc_bf16(128, UNIT, 0, 0);
-            const uint32_t idescV = ptx::instr_desc_bf16(128, DG, 0, 1);
+            const uint32_t idescV = ptx::instr_desc_bf16(128, kOnes ? DG + 16 : DG, 0, 1);
             // Q rows of the slot's latent block (K-major A operand); descriptor address fields are in 16-byte units
             const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ) +
                                    (uint64_t)(alternate ? 0 : j * kTile * G::RB / 16);
             const uint32_t gcol = tm + j * SLOT_COLS + c * 2 * HALF;        // the group's 128 columns
-            const uint32_t dcol = gcol + 2 * UNIT;                          // its accumulator
+            const uint32_t dcol = gcol + ACC_COL;                           // its accumulator
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 2);
             const int jobs = (nq - j + nslots - 1) / nslots;                // tiles this group works on
             const int units = 2 * jobs;
@@ -878,50 +1439,130 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // in hardware, so the issuing warp takes no issue slots from the softmax warps while it waits.
             int t_s = alternate ? j : 0, t_v = t_s;                         // tiles (relative to t_begin) of the next S / PV unit
             const int t_step = alternate ? 2 : 1;
-            auto issue_scores = [&](int n) -> bool {
-                const int s = t_s % kEncStages, w = n & 1;                  // w: which 32 tokens of the half; also the buffer
-                if (!ptx::mbar_wait(bar(KV_FULL + s), (t_s / kEncStages) & 1, abort_flag, kErrEncode | 3)) return false;
-                ptx::tc_fence_after();
-                // S_unit = Q_block K_unit^T: the unit's 32 token rows of the K tile are the B operand
-                const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES), 16, G::SBO, G::SWZ) +
-                                       (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
+            if constexpr (kFast) {
+                // The fast form's loop, with as few instructions of this thread per unit as it takes (they are on the
+                // critical path of the group: each waits for an issue slot among the softmax warps, and a tcgen05.mma or
+                // commit holds the thread for 50 to 130 cycles): descriptors are a base plus a stage and a unit offset;
+                // one wait per tile for the loads and one per unit for the weights; ONE commit per unit, behind the score
+                // MMA of the unit two further on, which tells the threads both that those scores are there and that the
+                // value MMAs before them (which read the buffer the scores went into) are done.
+                const uint32_t stage_step = (uint32_t)((2 * G::TILE_BYTES) >> 4), unit_step = (uint32_t)((UNIT * G::RB) >> 4);
+                const uint64_t kd0 = ptx::smem_desc(ptx::smem_u32(sKV), 16, G::SBO, G::SWZ) + (uint64_t)((c * HALF * G::RB) >> 4);
+                const uint32_t v0 = ptx::smem_u32(sKV + G::TILE_BYTES);
+                const uint64_t vd0 = ptx::smem_desc(v0, kOnes ? ptx::smem_u32(sOnes) - v0 : (uint32_t)G::SBO, G::SBO, G::SWZ) +
+                                     (uint64_t)((c * HALF * G::RB) >> 4);
+                // a stage further on, the V tile starts stage_step later and (kOnes) the ones tile is that much nearer (LBO: bits 16-29)
+                const uint64_t vstep = (uint64_t)stage_step - (kOnes ? ((uint64_t)stage_step << 16) : 0ull);
+                const uint32_t sfull = bar(S_FULL + 2 * g), pfull = bar(P_FULL + 2 * g);
+                // without kMaskBody only a last partial tile has padding; its scores get the bias MMA (see kMaskedScore)
+                const int bias_tile = (!kMaskBody && a.N % kTile != 0) ? a.tiles - 1 - t_begin : -1;
+                int ss = t_s % kEncStages, sp = (t_s / kEncStages) & 1, sv = ss;
+                auto scores = [&](int w) {                        // the scores of unit w of the S stream's tile, and the commit
+                    const uint64_t kd = kd0 + (uint64_t)(stage_step * (uint32_t)ss + unit_step * (uint32_t)w);
 #pragma unroll
-                for (int k = 0; k < DG / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
-                const int tile = t_begin + t_s;
-                if (!kDz && !kMaskBody && !(a.key_mask == nullptr && (tile + 1) * kTile <= a.N)) {
-                    // scores += ones x bias: padded tokens drop to kMaskedScore (see there)
-                    using GB = TileGeom<16>;
-                    const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)kEncStages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
-                    const uint64_t bdesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)s * SM::kBiasTile), 16, GB::SBO, GB::SWZ) +
-                                           (uint64_t)((c * HALF + w * UNIT) * GB::RB / 16);
-                    ptx::mma_ss(gcol + w * UNIT, odesc, bdesc, idescS, 1u);
+                    for (int k = 0; k < DG / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kd + 2 * k, idescS, k > 0);
+                    if (!kMaskBody && t_s == bias_tile) {
+                        using GB = TileGeom<16>;
+                        const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)kEncStages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
+                        const uint64_t bdesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)ss * SM::kBiasTile), 16, GB::SBO, GB::SWZ) +
+                                               (uint64_t)((c * HALF + w * UNIT) * GB::RB / 16);
+                        ptx::mma_ss(gcol + w * UNIT, odesc, bdesc, idescS, 1u);
+                    }
+                    ptx::mma_commit(sfull + 8 * w);
+                };
+                auto open_tile = [&]() -> bool {
+                    if (!ptx::mbar_wait(bar(KV_FULL + ss), (uint32_t)sp, abort_flag, kErrEncode | 3)) return false;
+                    ptx::tc_fence_after();
+                    return true;
+                };
+                auto next_s = [&]() {
+                    t_s += t_step;
+                    ss += t_step;
+                    if (ss >= kEncStages) { ss -= kEncStages; sp ^= 1; }
+                };
+                if (ok && jobs > 0 && (ok = open_tile())) {
+                    scores(0);
+                    scores(1);
+                    next_s();
                 }
-                ptx::mma_commit(bar(S_FULL + 2 * g + w));
-                if (w == 1) t_s += t_step;
-                return true;
-            };
-            for (int n = 0; ok && n < 2 && n < units; ++n) ok = issue_scores(n);
-            for (int n = 0; ok && n < units; ++n) {
-                const int w = n & 1, s = t_v % kEncStages;
-                if (!ptx::mbar_wait(bar(P_FULL + 2 * g + w), (n >> 1) & 1, abort_flag, kErrEncode | 4)) break;
-                ptx::tc_fence_after();
-                // acc += P_unit V_unit: V tile as the MN-major B operand, 16 token rows further on per k-step
-                const uint64_t vdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES),
-                                                      G::SBO, G::SBO, G::SWZ) + (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
+                for (int job = 0; ok && job < jobs; ++job) {
 #pragma unroll
-                for (int k = 0; k < UNIT / 16; ++k) {
-                    ptx::mma_ts(dcol, gcol + w * UNIT + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, (n > 0 || k > 0) ? 1u : 0u);
-                    if (kDz || kHiLo)    // the lo halves of the weights sit 16 columns further on
-                        ptx::mma_ts(dcol, gcol + w * UNIT + 16 + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, 1u);
+                    for (int w = 0; w < 2; ++w) {
+                        if (!ptx::mbar_spin(pfull + 8 * w, (uint32_t)(job & 1), abort_flag, kErrEncode | 4)) { ok = false; break; }
+                        ptx::tc_fence_after();
+                        const uint64_t vd = vd0 + vstep * (uint64_t)sv + (uint64_t)(unit_step * (uint32_t)w);
+#pragma unroll
+                        for (int k = 0; k < UNIT / 16; ++k) {
+                            ptx::mma_ts(dcol, gcol + w * UNIT + k * 8, vd + (uint64_t)(k * G::RB), idescV, (job > 0 || w > 0 || k > 0) ? 1u : 0u);
+                            if (kHiLo) ptx::mma_ts(dcol, gcol + w * UNIT + 16 + k * 8, vd + (uint64_t)(k * G::RB), idescV, 1u);
+                        }
+                        if (w == 1) {                             // the tile's last unit: one arrival per group
+                            ptx::mma_commit(bar(KV_EMPTY + sv));
+                            sv += t_step;
+                            if (sv >= kEncStages) sv -= kEncStages;
+                        }
+                        if (job + 1 < jobs) {                     // the same unit of the group's next tile, into the buffer just read
+                            if (w == 0 && !open_tile()) { ok = false; break; }
+                            scores(w);
+                            if (w == 1) next_s();
+                        }
+                    }
                 }
-                ptx::mma_commit(bar(PV_DONE + g));
-                if (w == 1) {                                               // the tile's last unit: one arrival per group
-                    ptx::mma_commit(bar(KV_EMPTY + s));
-                    t_v += t_step;
+                if (ok) ptx::mma_commit(bar(ACC_DONE + g));
+            } else {
+                int s_stage = t_s % kEncStages, s_phase = (t_s / kEncStages) & 1;   // stage and phase of the S stream's tile
+                auto issue_scores = [&](int n) -> bool {
+                    const int s = s_stage, w = n & 1;                        // w: which 32 tokens of the half; also the buffer
+                    if (!ptx::mbar_wait(bar(KV_FULL + s), s_phase, abort_flag, kErrEncode | 3)) return false;
+                    ptx::tc_fence_after();
+                    // S_unit = Q_block K_unit^T: the unit's 32 token rows of the K tile are the B operand
+                    const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES), 16, G::SBO, G::SWZ) +
+                                           (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
+#pragma unroll
+                    for (int k = 0; k < DG / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                    const int tile = t_begin + t_s;
+                    if (!kDz && !kMaskBody && !(a.key_mask == nullptr && (tile + 1) * kTile <= a.N)) {
+                        // scores += ones x bias: padded tokens drop to kMaskedScore (see there)
+                        using GB = TileGeom<16>;
+                        const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)kEncStages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
+                        const uint64_t bdesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)s * SM::kBiasTile), 16, GB::SBO, GB::SWZ) +
+                                               (uint64_t)((c * HALF + w * UNIT) * GB::RB / 16);
+                        ptx::mma_ss(gcol + w * UNIT, odesc, bdesc, idescS, 1u);
+                    }
+                    ptx::mma_commit(bar(S_FULL + 2 * g + w));
+                    if (w == 1) {
+                        t_s += t_step;
+                        s_stage += t_step;
+                        if (s_stage >= kEncStages) { s_stage -= kEncStages; s_phase ^= 1; }
+                    }
+                    return true;
+                };
+                for (int n = 0; ok && n < 2 && n < units; ++n) ok = issue_scores(n);
+                int v_stage = t_v % kEncStages;
+                for (int n = 0; ok && n < units; ++n) {
+                    const int w = n & 1, s = v_stage;
+                    if (!ptx::mbar_wait(bar(P_FULL + 2 * g + w), (n >> 1) & 1, abort_flag, kErrEncode | 4)) break;
+                    ptx::tc_fence_after();
+                    // acc += P_unit V_unit: V tile as the MN-major B operand, 16 token rows further on per k-step
+                    const uint64_t vdesc = ptx::smem_desc(ptx::smem_u32(sKV + (size_t)s * 2 * G::TILE_BYTES + G::TILE_BYTES),
+                                                          G::SBO, G::SBO, G::SWZ) + (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);
+#pragma unroll
+                    for (int k = 0; k < UNIT / 16; ++k) {
+                        ptx::mma_ts(dcol, gcol + w * UNIT + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, (n > 0 || k > 0) ? 1u : 0u);
+                        if (kDz || kHiLo)    // the lo halves of the weights sit 16 columns further on
+                            ptx::mma_ts(dcol, gcol + w * UNIT + 16 + k * 8, vdesc + (uint64_t)(k * G::RB), idescV, 1u);
+                    }
+                    ptx::mma_commit(bar(PV_DONE + g));
+                    if (w == 1) {                                           // the tile's last unit: one arrival per group
+                        ptx::mma_commit(bar(KV_EMPTY + s));
+                        t_v += t_step;
+                        v_stage += t_step;
+                        if (v_stage >= kEncStages) v_stage -= kEncStages;
+                    }
+                    if (n + 2 < units) ok = issue_scores(n + 2);
                 }
-                if (n + 2 < units) ok = issue_scores(n + 2);
+                if (ok) ptx::mma_commit(bar(ACC_DONE + g));
             }
-            if (ok) ptx::mma_commit(bar(ACC_DONE + g));
         }
     } else {
         const int g = (warp - kFirstSoftmaxWarp) >> 2;          // softmax group
@@ -929,7 +1570,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int row = ((warp & 3) << 5) + lane;               // TMEM lane = latent within the block
         const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
         const uint32_t gcol = tm + lane_addr + j * SLOT_COLS + c * 2 * HALF;   // the group's 128 columns
-        const uint32_t abase = gcol + 2 * UNIT;                               // its accumulator
+        const uint32_t abase = gcol + ACC_COL;                                // its accumulator
         const float2 sl2p = make_float2(a.sl2, a.sl2);
         float m_run = -INFINITY;
         float2 l2 = make_float2(0.f, 0.f);
@@ -1020,13 +1661,50 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             ++done;
             return true;
         };
+        // Fast form of a unit: weights 2^(s * sl2), no maximum, nothing to rescale.  kMasked as above; kPoly: half of
+        // the exponentials on the FMA pipe (never where padding sits in the scores as kMaskedScore).
+        auto unit_fast = [&](auto masked, auto poly, int t, int w) -> bool {
+            constexpr bool kMasked = decltype(masked)::value;
+            constexpr bool kPoly = decltype(poly)::value && !kHiLo;
+            uint32_t wv = 0xffffffffu;
+            if (kMasked) {
+                const int n = t * kTile + c * HALF + w * UNIT + lane;
+                wv = __ballot_sync(0xffffffffu, n < a.N && (a.key_mask == nullptr || a.key_mask[(size_t)b * a.N + n] != 0));
+            }
+            const uint32_t sbase = gcol + w * UNIT;
+            if (!warp_wait(bar(S_FULL + 2 * g + w), (done >> 1) & 1, abort_flag, kErrEncode | 5)) return false;
+            ptx::tc_fence_after();
+            uint32_t r[32], pk[16];
+            ptx::tmem_ld32(sbase, r);
+            ptx::tmem_wait_ld();
+            if (kHiLo) {
+                uint32_t pl[16];
+                exp_chunk_hilo<32, kMasked>(r, pk, pl, sl2p, make_float2(0.f, 0.f), l2, wv, false);
+                ptx::tmem_st16(sbase, pk);
+                ptx::tmem_st16(sbase + 16, pl);
+            } else {
+                exp_chunk_fast<32, kPoly, kMasked, kSumMode>(r, pk, sl2p, l2, wv);
+                ptx::tmem_st16(sbase, pk);
+            }
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(P_FULL + 2 * g + w));
+            ++done;
+            return true;
+        };
         if (j < nslots) {
             for (int q = j; ok && q < nq; q += nslots) {
                 const int t = t_begin + (alternate ? q : q / nslots);
-                const bool plain = !kMaskBody || (a.key_mask == nullptr && (t + 1) * kTile <= a.N);   // warp-uniform
+                const bool full = a.key_mask == nullptr && (t + 1) * kTile <= a.N;    // no padding in this tile (warp-uniform)
+                const bool plain = !kMaskBody || full;
 #pragma unroll 1
                 for (int w = 0; ok && w < 2; ++w) {             // the half's two units, on alternating buffers
                     if (kDz) ok = unit_dz(t, w);
+                    else if (kFast && kMaskBody) ok = plain ? unit_fast(std::false_type{}, std::true_type{}, t, w)
+                                                            : unit_fast(std::true_type{}, std::true_type{}, t, w);
+                    else if (kFast) ok = full ? unit_fast(std::false_type{}, std::true_type{}, t, w)
+                                              : unit_fast(std::false_type{}, std::false_type{}, t, w);
                     else if (kMaskBody && !plain) ok = unit(std::true_type{}, t, w);
                     else ok = unit(std::false_type{}, t, w);    // (without kMaskBody padding is in the scores already)
                 }
@@ -1044,11 +1722,18 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (done > 0) {
 #pragma unroll
             for (int dc = 0; dc < D / 16; ++dc) ptx::tmem_ld16(abase + second * D + dc * 16, acc + dc * 16);
+            if (kOnes) {                                        // column DG: the sum of the weights
+                uint32_t t8[8];
+                ptx::tmem_ld8(abase + DG, t8);
+                ptx::tmem_wait_ld();
+                l2 = make_float2(__uint_as_float(t8[0]), 0.f);
+            }
             ptx::tmem_wait_ld();
         } else {
 #pragma unroll
             for (int k = 0; k < D; ++k) acc[k] = 0u;
         }
+        if (kFast) m_run = (l2.x + l2.y > 0.f) ? 0.f : -INFINITY;   // weights relative to 2^0; a row with no valid token
         if (writes && m < M) {
             const long rows = (long)a.B * a.H * M;
             const int part = split * a.partials_per_split + (alternate ? 2 * j + c : c);

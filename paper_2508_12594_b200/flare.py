@@ -46,7 +46,8 @@ _SIGNATURES = {
     "flare_encode_partials": (ctypes.c_int, [_dp]),
     "flare_encode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "flare_encode_static_scratch": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
-    "flare_decode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "flare_decode": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "flare_set_path": (ctypes.c_int, [ctypes.c_int]),
     "flare_forward": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 13 + [_sz, _vp]),
     "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
@@ -163,13 +164,22 @@ def flare_encode_static_scratch(desc, Q, K, V, key_mask, Z, lse_enc, stream=None
     _raise(rc, "flare_encode_static_scratch")
 
 
-def flare_decode(desc, Q, K, Z, Y, lse_dec, stream=None):
+def flare_decode(desc, Q, K, Z, Y, lse_dec, workspace=None, stream=None):
     dt = K.dtype
     B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
     rc = load().flare_decode(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, (B, N, H, D)),
                              _ptr(Z, torch.float32, (B, H, M, D)), _ptr(Y, dt, (B, N, H, D)),
-                             _ptr(lse_dec, torch.float32, (B, N, H)), _stream(stream))
+                             _ptr(lse_dec, torch.float32, (B, N, H)), _ptr(workspace, torch.uint8),
+                             0 if workspace is None else workspace.numel(), _stream(stream))
     _raise(rc, "flare_decode")
+
+
+PATH_AUTO, PATH_EXACT, PATH_FAST = 0, 1, 2
+
+
+def flare_set_path(path: int):
+    """Which form of the bfloat16 forward kernels runs: PATH_AUTO, PATH_EXACT (running maximum) or PATH_FAST."""
+    _raise(load().flare_set_path(int(path)), "flare_set_path")
 
 
 def flare_forward(desc, Q, K, V, key_mask, Y, Z, lse_enc, lse_dec, workspace, stream=None):

@@ -60,8 +60,8 @@ def dev(t):
     return None if t is None else t.cuda()
 
 
-def gpu_forward(inp, scale=1.0, canary=False, stats=True):
-    """flare_forward on cuda:0.  With canary=True the outputs sit inside larger buffers whose margins must stay
+def gpu_forward(inp, scale=1.0, canary=False, stats=True, path=None):
+    """flare_forward on cuda:0.  path: None (the library's choice) or flare.PATH_EXACT / PATH_FAST for this call.  With canary=True the outputs sit inside larger buffers whose margins must stay
     untouched (checked here).  stats=False is the inference call the benchmark times: Z is asked for, the two
     log-sum-exp outputs are NULL (which selects other forms of the kernels).  Returns numpy float64
     dict(Y, Z, lse_enc, lse_dec), the last two None without stats."""
@@ -82,7 +82,12 @@ def gpu_forward(inp, scale=1.0, canary=False, stats=True):
     ldb, ld = padded((B, N, H), torch.float32, 777.0)
     if pad % 8 != 0:
         raise AssertionError("canary margin must keep 16-byte alignment")
-    flare.flare_forward(desc, Q, K, V, mask, Y, Z, le if stats else None, ld if stats else None, ws)
+    if path is not None:
+        flare.flare_set_path(path)
+    try:
+        flare.flare_forward(desc, Q, K, V, mask, Y, Z, le if stats else None, ld if stats else None, ws)
+    finally:
+        flare.flare_set_path(flare.PATH_AUTO)
     torch.cuda.synchronize()
     flare.flare_check(ws)
     if canary:

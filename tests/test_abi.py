@@ -60,7 +60,7 @@ def test_descriptor_validation_needs_no_device(lib):
     # null pointers are rejected before anything touches a device
     rc = lib.flare_encode(ctypes.byref(ok), None, None, None, None, None, None, None, 0, None)
     assert rc == flare.ERR_INVALID_ARG
-    rc = lib.flare_decode(ctypes.byref(flare.FlareDesc(1, 2, 8, 16, 12, 0, 1.0)), None, None, None, None, None, None)
+    rc = lib.flare_decode(ctypes.byref(flare.FlareDesc(1, 2, 8, 16, 12, 0, 1.0)), None, None, None, None, None, None, 0, None)
     assert rc == flare.ERR_UNSUPPORTED
 
 

@@ -28,18 +28,25 @@ SCALED = [
 
 
 # stats: the training call (Z and both log-sum-exp outputs) or the inference call the benchmark times (Z only; the
-# library then runs other forms of its kernels: single bfloat16 encode weights, no statistics written)
-STATS = pytest.mark.parametrize("stats", [True, False], ids=["train", "infer"])
+# library then runs other forms of its kernels: single bfloat16 encode weights, no statistics written).
+# path: the exact forms of the tensor-core kernels (running maximum) or the fast ones (none; polynomial exponentials),
+# forced, because left to itself the library takes the fast forms only for problems larger than these.
+STATS = pytest.mark.parametrize("stats,path", [(True, flare.PATH_EXACT), (False, flare.PATH_EXACT), (True, flare.PATH_FAST),
+                                               (False, flare.PATH_FAST)], ids=["train", "infer", "train-fast", "infer-fast"])
+
+
+def _mode(stats, path):
+    return ("train" if stats else "infer") + ("-fast" if path == flare.PATH_FAST else "")
 
 
 @pytest.mark.parametrize("w", SCALED, ids=lambda w: w.name)
 @pytest.mark.parametrize("paper_scale", [True, False], ids=["s=1", "s=1/sqrtD"])
 @STATS
-def test_scaled_down_workloads(oracle, w, paper_scale, stats):
+def test_scaled_down_workloads(oracle, w, paper_scale, stats, path):
     scale = 1.0 if paper_scale else w.D ** -0.5
     inp = workloads.make_inputs(w)
-    assert_forward_close(gpu_forward(inp, scale, canary=True, stats=stats), oracle_forward(oracle, inp, scale), w.dtype,
-                         f"{w.name} {'train' if stats else 'infer'}")
+    assert_forward_close(gpu_forward(inp, scale, canary=True, stats=stats, path=path), oracle_forward(oracle, inp, scale),
+                         w.dtype, f"{w.name} {_mode(stats, path)}")
 
 
 EDGE = [
@@ -80,11 +87,13 @@ EDGE = [
 
 @pytest.mark.parametrize("case", EDGE, ids=lambda c: "B{}H{}N{}M{}D{}{}m{}".format(*c))
 @STATS
-def test_edge_shapes(oracle, case, stats):
+def test_edge_shapes(oracle, case, stats, path):
     B, H, N, M, D, dtype, mf = case
+    if dtype == "f32" and path == flare.PATH_FAST:
+        pytest.skip("float32 inputs run on the CUDA cores: one form only")
     inp = workloads.make_random(B, H, N, M, D, dtype=dtype, seed=N + M, masked_fraction=mf, k_std=0.8)
-    assert_forward_close(gpu_forward(inp, canary=True, stats=stats), oracle_forward(oracle, inp), dtype,
-                         f"{case} {'train' if stats else 'infer'}")
+    assert_forward_close(gpu_forward(inp, canary=True, stats=stats, path=path), oracle_forward(oracle, inp), dtype,
+                         f"{case} {_mode(stats, path)}")
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -137,7 +146,7 @@ def test_encode_then_decode_equals_forward(oracle):
     Z2, le2 = torch.empty_like(Z1), torch.empty_like(le1)
     flare.flare_encode(desc, Q, K, V, mask, Z2, le2, ws)
     Y2, ld2 = torch.empty_like(Y1), torch.empty_like(ld1)
-    flare.flare_decode(desc, Q, K, Z2, Y2, ld2)
+    flare.flare_decode(desc, Q, K, Z2, Y2, ld2, flare.alloc_workspace(desc, flare.OP_DECODE))
     torch.cuda.synchronize()
     assert torch.equal(Z1, Z2) and torch.equal(le1, le2) and torch.equal(Y1, Y2) and torch.equal(ld1, ld2)
     # decode alone against the oracle's decode on the oracle's own Z
@@ -185,10 +194,11 @@ def test_error_paths_on_device():
 
 @pytest.mark.parametrize("k_std", [3.0, 8.0])
 @STATS
-def test_large_scores(oracle, k_std, stats):
-    """Scores up to +-170 at scale 1: the running maximum is subtracted before every exponential."""
+def test_large_scores(oracle, k_std, stats, path):
+    """Scores up to +-170 at scale 1: the running maximum is subtracted before every exponential; the fast forms find
+    their inputs out of range and hand over to the exact ones."""
     inp = workloads.make_random(1, 2, 700, 128, 16, dtype="bf16", seed=7, k_std=k_std)
-    got = gpu_forward(inp, canary=True, stats=stats)
+    got = gpu_forward(inp, canary=True, stats=stats, path=path)
     assert np.isfinite(got["Y"]).all() and np.isfinite(got["Z"]).all()
     assert_forward_close(got, oracle_forward(oracle, inp), "bf16", f"k_std={k_std}")
 
@@ -232,3 +242,24 @@ def test_bounded_wait_gives_up_and_reports(oracle):
     torch.cuda.synchronize()
     flare.flare_check(ws)
     assert rel_err(to_np64(Y), oracle_forward(oracle, inp)["Y"]) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("k_std,redo", [(0.5, False), (8.0, True)])
+def test_fast_forms_hand_over_only_when_out_of_range(oracle, k_std, redo):
+    """The flag words the fast forms raise (workspace header words 2 and 3: encode, decode) stay clear for ordinary
+    inputs and go up for scores beyond the range the fast forms are valid for; the result is right in both cases."""
+    inp = workloads.make_random(1, 2, 900, 128, 16, dtype="bf16", seed=11, k_std=k_std)
+    Q, K, V = dev(inp.Q), dev(inp.K), dev(inp.V)
+    desc = flare.make_desc(Q, K)
+    ws = flare.alloc_workspace(desc, flare.OP_FORWARD)
+    Y = torch.empty_like(K)
+    flare.flare_set_path(flare.PATH_FAST)
+    try:
+        flare.flare_forward(desc, Q, K, V, None, Y, None, None, None, ws)
+    finally:
+        flare.flare_set_path(flare.PATH_AUTO)
+    torch.cuda.synchronize()
+    words = ws[:16].view(torch.int32).cpu()
+    assert words[0] == 0 and bool(words[2]) == redo and bool(words[3]) == redo
+    from tests._util import assert_stored_close
+    assert_stored_close(to_np64(Y), oracle_forward(oracle, inp)["Y"], "bf16", f"fast forms, k_std={k_std}")

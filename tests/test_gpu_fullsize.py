@@ -55,8 +55,8 @@ def _forward_reference(oracle, w, inp):
     return _REF_CACHE[w.name]
 
 
+@pytest.mark.parametrize("stats", [True, False], ids=["train", "infer"])      # varies fastest: one oracle run per workload
 @pytest.mark.parametrize("w", FULL, ids=lambda w: w.name)
-@pytest.mark.parametrize("stats", [True, False], ids=["train", "infer"])
 def test_forward_full_size_sampled(oracle, w, stats):
     inp = workloads.make_inputs(w)
     Q, K, V, mask = dev(inp.Q), dev(inp.K), dev(inp.V), dev(inp.key_mask)
