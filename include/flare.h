@@ -59,7 +59,7 @@ typedef enum {
 } flare_status_t;
 
 enum { FLARE_DTYPE_F32 = 0, FLARE_DTYPE_BF16 = 1 };
-enum { FLARE_OP_ENCODE = 0, FLARE_OP_DECODE = 1, FLARE_OP_FORWARD = 2, FLARE_OP_BACKWARD = 3 };
+enum { FLARE_OP_ENCODE = 0, FLARE_OP_DECODE = 1, FLARE_OP_FORWARD = 2, FLARE_OP_BACKWARD = 3, FLARE_OP_SPECTRAL = 4 };
 
 typedef struct {
     int32_t B, H, N, M, D; /* batch, heads, tokens, latents per head, head width */
@@ -195,6 +195,30 @@ int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void 
 #define FLARE_STATIC_SCRATCH_BYTES (8u << 20)
 int flare_encode_static_scratch(const flare_desc_t *desc, const void *Q_lat, const void *K, const void *V,
                                 const uint8_t *key_mask, float *Z, float *lse_enc, flare_stream_t stream);
+
+/*
+ * Spectral analysis of the mixing matrix in O(M^2 N) (spectral-analysis appendix, Algorithm 1).  Per (b, h) the
+ * N x N mixing matrix W = W_dec W_enc has rank at most M, and its non-zero eigenvalues are those of the M x M
+ * matrix G = J J^T, J = L_M^{1/2} A L_N^{1/2}, A = exp(scale Q K^T), L_M = diag(1 / row sums of A),
+ * L_N = diag(1 / column sums of A) (the appendix once writes "J^T J" for the M x M matrix; the algorithm's steps
+ * fix it as J J^T).  flare_spectral_gram forms G [B, H, M, M] float32 from Q_lat, K and the two log-sum-exp
+ * outputs of flare_forward on the same Q_lat and K (lse_enc = log row sums, lse_dec = log column sums, both of
+ * all tokens: no key mask), J[m,n] = exp(score - lse_enc[m]/2 - lse_dec[n]/2): one pass over the tokens, nothing of
+ * size M x N is written.  bfloat16 inputs with M <= 128 and D in {16, 32} run on the tensor cores; everything else on
+ * the CUDA cores.  Workspace: flare_workspace_bytes(desc, FLARE_OP_SPECTRAL).
+ */
+int flare_spectral_gram(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *lse_enc,
+                        const float *lse_dec, float *G, void *workspace, size_t workspace_bytes, flare_stream_t stream);
+
+/*
+ * The M x M symmetric eigenproblems of Algorithm 1 (its step "U Sigma^2 U^T = J J^T"), O(M^3) each and off the hot
+ * path: cyclic Jacobi rotations, one thread block per matrix.  G [matrices, M, M] float32 is destroyed;
+ * eigenvalues [matrices, M] come out in descending order; U [matrices, M, M] (may be NULL) gets the eigenvectors as
+ * columns, in the same order.  sweeps <= 0 means the default (12).  M <= 1024.  (The eigenvectors of W itself,
+ * L_N^{1/2} J^T U Sigma^{-1}, are N x M and are not formed.)
+ */
+int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues, float *U, int32_t sweeps,
+                       flare_stream_t stream);
 
 /*
  * After the stream has been synchronised: FLARE_OK, or FLARE_ERR_TIMEOUT if a kernel of the last call that

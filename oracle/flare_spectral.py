@@ -19,8 +19,8 @@ from __future__ import annotations
 import numpy as np
 
 
-def eig_from_qk(Q_h, K_h, scale: float = 1.0):
-    """Q_h [M, D], K_h [N, D] of one head -> (eigenvalues [M] descending, eigenvectors [N, M])."""
+def gram_from_qk(Q_h, K_h, scale: float = 1.0):
+    """Steps 1-4 of Algorithm 1 and the M x M matrix of step 5: Q_h [M, D], K_h [N, D] -> (J J^T [M, M], J [M, N], L_N [N])."""
     Q_h = np.asarray(Q_h, dtype=np.float64)
     K_h = np.asarray(K_h, dtype=np.float64)
     S = scale * (Q_h @ K_h.T)
@@ -28,7 +28,13 @@ def eig_from_qk(Q_h, K_h, scale: float = 1.0):
     L_N = 1.0 / A.sum(axis=0)
     L_M = 1.0 / A.sum(axis=1)
     J = np.sqrt(L_M)[:, None] * A * np.sqrt(L_N)[None, :]
-    sig2, U = np.linalg.eigh(J @ J.T)
+    return J @ J.T, J, L_N
+
+
+def eig_from_qk(Q_h, K_h, scale: float = 1.0):
+    """Q_h [M, D], K_h [N, D] of one head -> (eigenvalues [M] descending, eigenvectors [N, M])."""
+    JJt, J, L_N = gram_from_qk(Q_h, K_h, scale)
+    sig2, U = np.linalg.eigh(JJt)
     order = np.argsort(sig2)[::-1]
     sig2, U = sig2[order], U[:, order]
     sigma = np.sqrt(np.clip(sig2, 0.0, None))

@@ -13,6 +13,7 @@
 #include "flare_bwd.cuh"
 #include "flare_tc.cuh"
 #include "flare_bwd_tc.cuh"
+#include "flare_spectral.cuh"
 
 using namespace flare;
 
@@ -857,6 +858,67 @@ int launches_for(const flare_desc_t *d, int op, int sms) {
     }
 }
 
+// ---- spectral analysis (Algorithm 1 of the paper's spectral appendix)
+bool spectral_on_tensor_cores(const flare_desc_t *d) {
+    return d->dtype == FLARE_DTYPE_BF16 && d->scale > 0.f && (d->D == 16 || d->D == 32) && d->M <= kTile && d->M % 16 == 0;
+}
+int spectral_splits(const flare_desc_t *d, int sms) {
+    const int tiles = (d->N + kTile - 1) / kTile;
+    long s = sms / ((long)d->B * d->H);
+    if (s < 1) s = 1;
+    if (s > tiles) s = tiles;
+    return (int)s;
+}
+size_t spectral_bytes(const flare_desc_t *d, int sms) {
+    if (!spectral_on_tensor_cores(d)) return kHeaderBytes;
+    return kHeaderBytes + align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * d->B * d->H * kTile * kTile);
+}
+
+template <int D>
+int launch_spectral_gram_tc(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *lse_enc,
+                            const float *lse_dec, float *G, char *ws, cudaStream_t st) {
+    CUtensorMap tmK, tmQ;
+    int rc;
+    if ((rc = make_token_map(&tmK, K, d, kTile, D)) != FLARE_OK) return rc;
+    if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
+    static std::atomic<uint64_t> smem_opt_in{0};
+    if (int rc_attr = ensure_big_smem(spectral_gram_tc_kernel<D>, smem_opt_in, 227 * 1024)) return rc_attr;
+    SpectralArgs a;
+    a.Q = static_cast<const __nv_bfloat16 *>(Q);
+    a.lse_enc = lse_enc; a.lse_dec = lse_dec;
+    a.part = reinterpret_cast<float *>(ws + kHeaderBytes);
+    a.status = reinterpret_cast<uint32_t *>(ws);
+    a.B = d->B; a.H = d->H; a.N = d->N; a.M = d->M;
+    a.sl2 = d->scale * kLog2e;
+    a.tiles = (d->N + kTile - 1) / kTile;
+    a.splits = spectral_splits(d, sms);
+    spectral_gram_tc_kernel<D><<<dim3(a.splits, d->H, d->B), kTcThreads, SpectralSmem<D>::total, st>>>(tmK, tmQ, a);
+    FLARE_CUDA(cudaGetLastError());
+    const long n = (long)d->B * d->H * d->M * d->M;
+    spectral_gram_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.part, G, a.splits, (long)d->B * d->H, d->M);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+template <typename T>
+int launch_spectral_gram_simt(const flare_desc_t *d, const void *Q, const void *K, const float *lse_enc, const float *lse_dec,
+                              float *G, cudaStream_t st) {
+    const int tm = (d->M + 15) / 16;
+    dim3 grid(tm * tm, d->H, d->B);
+#define FLARE_CASE(DD)                                                                                                   \
+    case DD:                                                                                                             \
+        spectral_gram_simt_kernel<T, DD><<<grid, 256, 0, st>>>((const T *)Q, (const T *)K, lse_enc, lse_dec, G, d->B, d->H, \
+                                                              d->N, d->M, d->scale);                                     \
+        break;
+    switch (d->D) {
+        FLARE_CASE(4) FLARE_CASE(8) FLARE_CASE(16) FLARE_CASE(32) FLARE_CASE(64)
+        default: return FLARE_ERR_UNSUPPORTED;
+    }
+#undef FLARE_CASE
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -897,6 +959,7 @@ size_t flare_workspace_bytes(const flare_desc_t *desc, int op) {
         case FLARE_OP_FORWARD:
             return make_layout(partials_for(desc, device_info().sms), rows, desc->D, true).total + decode_range_bytes(desc);
         case FLARE_OP_BACKWARD: return bwd_layout(desc, device_info().sms).total;
+        case FLARE_OP_SPECTRAL: return spectral_bytes(desc, device_info().sms);
         default: return 0;
     }
 }
@@ -1016,6 +1079,40 @@ int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void 
                        workspace_bytes, stream);
     if (rc != FLARE_OK) return rc;
     FLARE_CUDA(cudaMemcpyAsync(hY, dY, tb, cudaMemcpyDeviceToHost, st));
+    return FLARE_OK;
+}
+
+int flare_spectral_gram(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *lse_enc,
+                        const float *lse_dec, float *G, void *workspace, size_t workspace_bytes, flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    const void *ptrs[] = {Q_lat, K, lse_enc, lse_dec, G, workspace};
+    for (const void *p : ptrs)
+        if (p == nullptr || !aligned16(p)) return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    const int sms = device_info().sms;
+    if (workspace_bytes < spectral_bytes(desc, sms)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    FLARE_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, st));
+    if (spectral_on_tensor_cores(desc) && use_tc(desc)) {
+        char *ws = static_cast<char *>(workspace);
+        return desc->D == 16 ? launch_spectral_gram_tc<16>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st)
+                             : launch_spectral_gram_tc<32>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st);
+    }
+    return desc->dtype == FLARE_DTYPE_F32 ? launch_spectral_gram_simt<float>(desc, Q_lat, K, lse_enc, lse_dec, G, st)
+                                          : launch_spectral_gram_simt<__nv_bfloat16>(desc, Q_lat, K, lse_enc, lse_dec, G, st);
+}
+
+int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues, float *U, int32_t sweeps, flare_stream_t stream) {
+    if (matrices <= 0 || M <= 0 || M > 1024 || !G || !eigenvalues) return FLARE_ERR_INVALID_ARG;
+    if (!aligned16(G) || !aligned16(eigenvalues) || (U && !aligned16(U))) return FLARE_ERR_INVALID_ARG;
+    int rc = require_device();
+    if (rc != FLARE_OK) return rc;
+    if (sweeps <= 0) sweeps = 12;
+    const int pairs = ((M + 1) & ~1) / 2;
+    const size_t shmem = sizeof(float) * (4 * (size_t)pairs + M);
+    spectral_jacobi_kernel<<<(unsigned)matrices, 256, shmem, (cudaStream_t)stream>>>(G, eigenvalues, U, M, sweeps);
+    FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 

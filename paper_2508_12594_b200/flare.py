@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libflare.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(7)
 DTYPE_F32, DTYPE_BF16 = 0, 1
-OP_ENCODE, OP_DECODE, OP_FORWARD, OP_BACKWARD = range(4)
+OP_ENCODE, OP_DECODE, OP_FORWARD, OP_BACKWARD, OP_SPECTRAL = range(5)
 
 
 class FlareDesc(ctypes.Structure):
@@ -52,6 +52,8 @@ _SIGNATURES = {
     "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 13 + [_sz, _vp]),
     "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
     "flare_check": (ctypes.c_int, [_vp, _vp]),
+    "flare_spectral_gram": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "flare_spectral_eig": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32, _vp, _vp, _vp, ctypes.c_int32, _vp]),
     "flare_launch_count": (ctypes.c_int, [_dp, ctypes.c_int]),
     "flare_selftest_wait": (ctypes.c_int, [_vp, ctypes.c_uint64, _vp]),
 }
@@ -230,6 +232,25 @@ def flare_launch_count(desc: FlareDesc, op: int) -> int:
 
 def flare_selftest_wait(workspace, budget_ns: int, stream=None):
     _raise(load().flare_selftest_wait(_ptr(workspace, torch.uint8), int(budget_ns), _stream(stream)), "flare_selftest_wait")
+
+
+def flare_spectral_gram(desc, Q, K, lse_enc, lse_dec, G, workspace, stream=None):
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    rc = load().flare_spectral_gram(ctypes.byref(desc), _ptr(Q, dt, (H, M, D)), _ptr(K, dt, (B, N, H, D)),
+                                    _ptr(lse_enc, torch.float32, (B, H, M)), _ptr(lse_dec, torch.float32, (B, N, H)),
+                                    _ptr(G, torch.float32, (B, H, M, M)), _ptr(workspace, torch.uint8), workspace.numel(),
+                                    _stream(stream))
+    _raise(rc, "flare_spectral_gram")
+
+
+def flare_spectral_eig(G, eigenvalues, U=None, sweeps=0, stream=None):
+    """G [..., M, M] float32 (destroyed) -> eigenvalues [..., M] descending, U [..., M, M] eigenvectors as columns."""
+    M = G.shape[-1]
+    matrices = G.numel() // (M * M)
+    rc = load().flare_spectral_eig(matrices, M, _ptr(G, torch.float32), _ptr(eigenvalues, torch.float32),
+                                   _ptr(U, torch.float32), int(sweeps), _stream(stream))
+    _raise(rc, "flare_spectral_eig")
 
 
 def forward(Q, K, V, key_mask=None, scale=1.0, want_stats=False, stream=None):

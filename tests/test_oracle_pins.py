@@ -248,6 +248,21 @@ def test_backward_value_gradient_sums(oracle):
     assert (g["dV"][mask == 0] == 0).all()
 
 
+def test_gram_of_algorithm_one_against_the_two_softmax_matrices(oracle):
+    """J = L_M^{1/2} A L_N^{1/2} has J[m,n]^2 = W_enc[m,n] W_dec[n,m] (A / row sum and A / column sum are the two softmax
+    matrices), so J J^T can be rebuilt from the oracle's dense W_enc and W_dec, which come from other code."""
+    from oracle import flare_spectral
+    B, H, N, M, D = 1, 2, 70, 6, 4
+    Q, K, V, _, _ = _np(workloads.make_random(B, H, N, M, D, seed=47))
+    for h in range(H):
+        We, Wd, _ = oracle.mixing_matrices(Q, K, 0, h, scale=0.6)
+        J = np.sqrt(We * Wd.T)
+        G, J_alg, _ = flare_spectral.gram_from_qk(Q[h], K[0, :, h], 0.6)
+        np.testing.assert_allclose(J_alg, J, rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(G, J @ J.T, rtol=1e-12)
+        np.testing.assert_allclose(np.trace(G), np.sum(We * Wd.T), rtol=1e-12)
+
+
 def test_backward_rows_matches_full(oracle):
     """The sampled-rows backward is the full backward restricted to the listed tokens, bit for bit (dQ and dZ are
     full reductions in both)."""
