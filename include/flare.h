@@ -197,6 +197,29 @@ int flare_encode_static_scratch(const flare_desc_t *desc, const void *Q_lat, con
                                 const uint8_t *key_mask, float *Z, float *lse_enc, flare_stream_t stream);
 
 /*
+ * Two variants of the mixer that the paper discusses and sets aside (both as entry points of their own; the plain
+ * calls above are the method as the paper uses it):
+ *   shared_latents != 0   all heads use ONE latent sequence (the "shared vs independent latents" ablation of the
+ *                         paper's ablation appendix): Q_enc, Q_dec, dQ_enc, dQ_dec are [M, D] instead of [H, M, D].
+ *   Q_dec != NULL         separate latent queries for the two stages (the "asymmetric" remark of the
+ *                         design-principles appendix): encode scores are Q_enc K^T, decode scores K Q_dec^T.
+ *                         NULL means the symmetric operator (Q_dec = Q_enc); dQ_dec must be NULL exactly then.
+ * Both are built from the kernels of the plain calls: a shared sequence is copied out to all heads in the workspace
+ * and its gradient summed over the heads; with separate queries the backward runs its two per-token passes twice,
+ * once per set of queries, each time with the other stage's weights switched off (its log-sum-exp rows set to
+ * +infinity), and adds the two parts of dK.  Workspace: flare_variant_workspace_bytes.  Everything else as in
+ * flare_forward / flare_backward.
+ */
+size_t flare_variant_workspace_bytes(const flare_desc_t *desc, int op, int shared_latents, int separate_decode_queries);
+int flare_forward_variant(const flare_desc_t *desc, int shared_latents, const void *Q_enc, const void *Q_dec, const void *K,
+                          const void *V, const uint8_t *key_mask, void *Y, float *Z, float *lse_enc, float *lse_dec,
+                          void *workspace, size_t workspace_bytes, flare_stream_t stream);
+int flare_backward_variant(const flare_desc_t *desc, int shared_latents, const void *Q_enc, const void *Q_dec, const void *K,
+                           const void *V, const uint8_t *key_mask, const void *Y, const void *dY, const float *Z,
+                           const float *lse_enc, const float *lse_dec, float *dQ_enc, float *dQ_dec, void *dK, void *dV,
+                           void *workspace, size_t workspace_bytes, flare_stream_t stream);
+
+/*
  * Spectral analysis of the mixing matrix in O(M^2 N) (spectral-analysis appendix, Algorithm 1).  Per (b, h) the
  * N x N mixing matrix W = W_dec W_enc has rank at most M, and its non-zero eigenvalues are those of the M x M
  * matrix G = J J^T, J = L_M^{1/2} A L_N^{1/2}, A = exp(scale Q K^T), L_M = diag(1 / row sums of A),

@@ -302,6 +302,62 @@ void flare_oracle_backward_rows(int B, int H, int N, int M, int D, double scale,
     backward_impl(B, H, N, M, D, scale, Q, K, V, key_mask, dY, rows, nrows, dQ, dK_rows, dV_rows, dZ_out);
 }
 
+/*
+ * Backward of the mixer with separate latent queries for the two stages (the "asymmetric" variant the paper's
+ * design-principles appendix mentions and sets aside): encode scores q^e_m . k_n, decode scores k_n . q^d_m,
+ *   Z = softmax(s Qe K^T) V,   Y = softmax(s K Qd^T) Z.
+ * The chain rule as above, with each stage's weights and score gradient on its own queries:
+ *   dSd[m,n] = W_dec[n,m] (dY_n . Z_m - dY_n . Y_n),      dSe[m,n] = W_enc[m,n] (dZ_m . V_n - dZ_m . Z_m),
+ *   dQd_m = s sum_n dSd[m,n] K_n,   dQe_m = s sum_n dSe[m,n] K_n,   dK_n = s sum_m (dSd[m,n] Qd_m + dSe[m,n] Qe_m).
+ * Outputs: dQe, dQd [H, M, D] (summed over the batch), dK, dV [B, N, H, D].  Dense loops; small cases.
+ */
+void flare_oracle_backward_asym(int B, int H, int N, int M, int D, double scale, const double *Qe, const double *Qd,
+                                const double *K, const double *V, const uint8_t *key_mask, const double *dY, double *dQe,
+                                double *dQd, double *dK, double *dV) {
+    size_t nZ = (size_t)B * H * M * D, nT = (size_t)B * N * H * D;
+    double *Z = (double *)malloc(sizeof(double) * nZ);
+    double *dZ = (double *)calloc(nZ, sizeof(double));
+    double *Y = (double *)malloc(sizeof(double) * nT);
+    double *le = (double *)malloc(sizeof(double) * (size_t)B * H * M);
+    double *ld = (double *)malloc(sizeof(double) * (size_t)B * N * H);
+    flare_oracle_encode(B, H, N, M, D, scale, Qe, K, V, key_mask, Z, le);
+    flare_oracle_decode(B, H, N, M, D, scale, Qd, K, Z, Y, ld);
+    for (size_t i = 0; i < (size_t)H * M * D; ++i) dQe[i] = 0.0, dQd[i] = 0.0;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            for (int m = 0; m < M; ++m) {                       /* dZ_m = sum_n W_dec[n,m] dY_n */
+                double *dz = dZ + IDX_Z(b, h, m);
+                for (int n = 0; n < N; ++n) {
+                    double wdec = exp(scale * dot(K + IDX_T(b, n, h), Qd + IDX_Q(h, m), D) - ld[((size_t)b * N + n) * H + h]);
+                    for (int d = 0; d < D; ++d) dz[d] += wdec * dY[IDX_T(b, n, h) + d];
+                }
+            }
+            for (int n = 0; n < N; ++n) {
+                const double *k = K + IDX_T(b, n, h), *v = V + IDX_T(b, n, h), *dy = dY + IDX_T(b, n, h);
+                double *dk = dK + IDX_T(b, n, h), *dv = dV + IDX_T(b, n, h);
+                int valid = !(key_mask && !key_mask[(size_t)b * N + n]);
+                double delta_d = dot(dy, Y + IDX_T(b, n, h), D);
+                for (int d = 0; d < D; ++d) dk[d] = 0.0, dv[d] = 0.0;
+                for (int m = 0; m < M; ++m) {
+                    const double *qe = Qe + IDX_Q(h, m), *qd = Qd + IDX_Q(h, m);
+                    const double *z = Z + IDX_Z(b, h, m), *dz = dZ + IDX_Z(b, h, m);
+                    double lem = le[((size_t)b * H + h) * M + m];
+                    double wdec = exp(scale * dot(k, qd, D) - ld[((size_t)b * N + n) * H + h]);
+                    double wenc = (valid && lem != -INFINITY) ? exp(scale * dot(k, qe, D) - lem) : 0.0;
+                    double dSd = wdec * (dot(dy, z, D) - delta_d);
+                    double dSe = wenc * (dot(dz, v, D) - dot(dz, z, D));
+                    for (int d = 0; d < D; ++d) {
+                        dv[d] += wenc * dz[d];
+                        dk[d] += scale * (dSd * qd[d] + dSe * qe[d]);
+                        dQd[IDX_Q(h, m) + d] += scale * dSd * k[d];
+                        dQe[IDX_Q(h, m) + d] += scale * dSe * k[d];
+                    }
+                }
+            }
+        }
+    free(Z); free(dZ); free(Y); free(le); free(ld);
+}
+
 int flare_oracle_max_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

@@ -152,3 +152,16 @@ def backward_rows(Q, K, V, dY, rows, key_mask=None, scale=1.0):
                                        rows.ctypes.data_as(_i64p), len(rows), dQ.ctypes.data_as(_dp),
                                        dK.ctypes.data_as(_dp), dV.ctypes.data_as(_dp), dZ.ctypes.data_as(_dp))
     return dict(dQ=dQ, dK_rows=dK, dV_rows=dV, dZ=dZ)
+
+
+def backward_asym(Qe, Qd, K, V, dY, key_mask=None, scale=1.0):
+    """Gradients of sum(Y * dY) for the variant with separate encode and decode queries (Qe, Qd [H,M,D]).
+    Returns dict(dQe, dQd [H,M,D], dK, dV [B,N,H,D]).  Dense and single-threaded: small cases only."""
+    B, H, N, M, D = _dims(Qe, K)
+    Qe, pqe = _d(Qe); Qd, pqd = _d(Qd); K, pk = _d(K); V, pv = _d(V); dY, pdy = _d(dY)
+    mk, pm = _mask(key_mask, B, N)
+    dQe = np.empty((H, M, D)); dQd = np.empty((H, M, D)); dK = np.empty((B, N, H, D)); dV = np.empty((B, N, H, D))
+    _load().flare_oracle_backward_asym(B, H, N, M, D, ctypes.c_double(scale), pqe, pqd, pk, pv, pm, pdy,
+                                       dQe.ctypes.data_as(_dp), dQd.ctypes.data_as(_dp), dK.ctypes.data_as(_dp),
+                                       dV.ctypes.data_as(_dp))
+    return dict(dQe=dQe, dQd=dQd, dK=dK, dV=dV)

@@ -579,7 +579,9 @@ BwdLayout bwd_layout(const flare_desc_t *d, int sms) {
 template <typename T, int D>
 int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V,
                          const uint8_t *mask, const void *Y, const void *dY, const float *Z, const float *lse_enc,
-                         const float *lse_dec, float *dQ, void *dK, void *dV, char *ws, cudaStream_t st) {
+                         const float *lse_dec, float *dQ, void *dK, void *dV, char *ws, cudaStream_t st,
+                         bool skip_pass_a = false) {
+    // skip_pass_a: dZ and de are already in the workspace (the second of the two runs of the separate-queries variant)
     const BwdLayout w = bwd_layout(d, sms);
     float *part = reinterpret_cast<float *>(ws + w.part);
     float *dZ = reinterpret_cast<float *>(ws + w.dz);
@@ -590,9 +592,9 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
     const SimtPlan pa = simt_plan(d, sms), pb = bwd_dq_plan(d, sms);
     FLARE_CUDA(cudaMemsetAsync(ws, 0, kHeaderBytes, st));
     int dz_parts = pa.P;
-    bool dz_on_tc = false;
+    bool dz_on_tc = skip_pass_a;
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-        if (bwd_dz_on_tensor_cores(d)) {
+        if (!skip_pass_a && bwd_dz_on_tensor_cores(d)) {
             const TcEncodePlan tp = tc_encode_plan(d, sms);
             uint32_t *status = reinterpret_cast<uint32_t *>(ws);
             int rc;
@@ -615,10 +617,12 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
             (const T *)Q, (const T *)K, (const T *)dY, lse_dec, part, d->B, d->H, d->N, d->M, pa.LM, pa.chunk, d->scale);
         FLARE_CUDA(cudaGetLastError());
     }
-    bwd_dz_reduce_kernel<<<(unsigned)((rows * d->D + 255) / 256), 256, 0, st>>>(part, dZ, dz_parts, rows, d->D);
-    FLARE_CUDA(cudaGetLastError());
-    bwd_de_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(dZ, Z, de, rows, d->D);
-    FLARE_CUDA(cudaGetLastError());
+    if (!skip_pass_a) {
+        bwd_dz_reduce_kernel<<<(unsigned)((rows * d->D + 255) / 256), 256, 0, st>>>(part, dZ, dz_parts, rows, d->D);
+        FLARE_CUDA(cudaGetLastError());
+        bwd_de_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(dZ, Z, de, rows, d->D);
+        FLARE_CUDA(cudaGetLastError());
+    }
     bool tok_on_tc = false;
     if constexpr (std::is_same<T, __nv_bfloat16>::value && D <= 32) {
         constexpr int DK = D < 16 ? 16 : D;                     // width the kernels multiply (D < 16: narrow forms)
@@ -680,13 +684,13 @@ int launch_backward_simt(const flare_desc_t *d, int sms, const void *Q, const vo
 template <typename T>
 int backward_simt(const flare_desc_t *d, int sms, const void *Q, const void *K, const void *V, const uint8_t *mask,
                   const void *Y, const void *dY, const float *Z, const float *lse_enc, const float *lse_dec, float *dQ,
-                  void *dK, void *dV, char *ws, cudaStream_t st) {
+                  void *dK, void *dV, char *ws, cudaStream_t st, bool skip_pass_a = false) {
     switch (d->D) {
-        case 4: return launch_backward_simt<T, 4>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
-        case 8: return launch_backward_simt<T, 8>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
-        case 16: return launch_backward_simt<T, 16>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
-        case 32: return launch_backward_simt<T, 32>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
-        case 64: return launch_backward_simt<T, 64>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st);
+        case 4: return launch_backward_simt<T, 4>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st, skip_pass_a);
+        case 8: return launch_backward_simt<T, 8>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st, skip_pass_a);
+        case 16: return launch_backward_simt<T, 16>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st, skip_pass_a);
+        case 32: return launch_backward_simt<T, 32>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st, skip_pass_a);
+        case 64: return launch_backward_simt<T, 64>(d, sms, Q, K, V, mask, Y, dY, Z, lse_enc, lse_dec, dQ, dK, dV, ws, st, skip_pass_a);
         default: return FLARE_ERR_UNSUPPORTED;
     }
 }
@@ -919,6 +923,66 @@ int launch_spectral_gram_simt(const flare_desc_t *d, const void *Q, const void *
     return FLARE_OK;
 }
 
+// ---- variants of the mixer: one latent sequence shared by all heads; separate latent queries for decode
+
+template <typename T>
+__global__ void expand_heads_kernel(const T *__restrict__ src, T *__restrict__ dst, long per_head, int H) {
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= per_head * H) return;
+    dst[i] = src[i % per_head];
+}
+__global__ void sum_heads_kernel(const float *__restrict__ src, float *__restrict__ dst, long per_head, int H) {
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= per_head) return;
+    float s = 0.f;
+    for (int h = 0; h < H; ++h) s += src[(size_t)h * per_head + i];
+    dst[i] = s;
+}
+__global__ void fill_kernel(float *__restrict__ dst, long n, float v) {
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = v;
+}
+template <typename T>
+__global__ void add_into_kernel(T *__restrict__ dst, const T *__restrict__ other, long n) {
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    T out;
+    from_f32(out, to_f32(dst[i]) + to_f32(other[i]));
+    dst[i] = out;
+}
+
+struct VariantLayout {
+    size_t qe, qd, dq_full, dq2_full, inf_enc, inf_dec, dk2, total;   // offsets behind the operation's own workspace
+};
+// Scratch of the variant entry points, behind the workspace of the plain operation (base bytes).
+VariantLayout variant_layout(const flare_desc_t *d, int op, int shared, int separate, size_t base) {
+    VariantLayout v{};
+    const size_t e = d->dtype == FLARE_DTYPE_F32 ? 4 : 2;
+    const size_t q = align_up((size_t)d->H * d->M * d->D * e), qf = align_up((size_t)d->H * d->M * d->D * 4);
+    size_t off = align_up(base);
+    v.qe = off; if (shared) off += q;
+    v.qd = off; if (shared && separate) off += q;
+    if (op == FLARE_OP_BACKWARD) {
+        v.dq_full = off; if (shared) off += qf;
+        v.dq2_full = off; if (shared && separate) off += qf;
+        v.inf_enc = off; if (separate) off += align_up(sizeof(float) * (size_t)d->B * d->H * d->M);
+        v.inf_dec = off; if (separate) off += align_up(sizeof(float) * (size_t)d->B * d->N * d->H);
+        v.dk2 = off; if (separate) off += align_up((size_t)d->B * d->N * d->H * d->D * e);
+    }
+    v.total = off;
+    return v;
+}
+
+int expand_heads(const flare_desc_t *d, const void *src, void *dst, cudaStream_t st) {
+    const long per = (long)d->M * d->D, n = per * d->H;
+    if (d->dtype == FLARE_DTYPE_F32)
+        expand_heads_kernel<float><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const float *)src, (float *)dst, per, d->H);
+    else
+        expand_heads_kernel<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)src, (__nv_bfloat16 *)dst, per, d->H);
+    FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1079,6 +1143,111 @@ int flare_forward_host(const flare_desc_t *desc, const void *hQ_lat, const void 
                        workspace_bytes, stream);
     if (rc != FLARE_OK) return rc;
     FLARE_CUDA(cudaMemcpyAsync(hY, dY, tb, cudaMemcpyDeviceToHost, st));
+    return FLARE_OK;
+}
+
+size_t flare_variant_workspace_bytes(const flare_desc_t *desc, int op, int shared_latents, int separate_decode_queries) {
+    if (op != FLARE_OP_FORWARD && op != FLARE_OP_BACKWARD) return 0;
+    const size_t base = flare_workspace_bytes(desc, op);
+    if (base == 0) return 0;
+    return variant_layout(desc, op, shared_latents, separate_decode_queries, base).total;
+}
+
+int flare_forward_variant(const flare_desc_t *desc, int shared_latents, const void *Q_enc, const void *Q_dec, const void *K,
+                          const void *V, const uint8_t *key_mask, void *Y, float *Z, float *lse_enc, float *lse_dec,
+                          void *workspace, size_t workspace_bytes, flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    if (!Q_enc || !K || !V || !Y || !workspace) return FLARE_ERR_INVALID_ARG;
+    const void *ptrs[] = {Q_enc, Q_dec, K, V, Y, Z, lse_enc, lse_dec, workspace};
+    for (const void *p : ptrs)
+        if (p != nullptr && !aligned16(p)) return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    const size_t base = flare_workspace_bytes(desc, FLARE_OP_FORWARD);
+    const VariantLayout v = variant_layout(desc, FLARE_OP_FORWARD, shared_latents, Q_dec != nullptr, base);
+    if (workspace_bytes < v.total) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = static_cast<char *>(workspace);
+    const void *qe = Q_enc, *qd = Q_dec ? Q_dec : Q_enc;
+    if (shared_latents) {
+        if ((rc = expand_heads(desc, Q_enc, ws + v.qe, st)) != FLARE_OK) return rc;
+        qe = ws + v.qe;
+        qd = qe;
+        if (Q_dec) {
+            if ((rc = expand_heads(desc, Q_dec, ws + v.qd, st)) != FLARE_OK) return rc;
+            qd = ws + v.qd;
+        }
+    }
+    const WorkspaceLayout w = make_layout(partials_for(desc, device_info().sms), (long)desc->B * desc->H * desc->M, desc->D, true);
+    if (Z == nullptr) Z = reinterpret_cast<float *>(ws + w.z);
+    if ((rc = encode_impl(desc, qe, K, V, key_mask, Z, lse_enc, workspace, st)) != FLARE_OK) return rc;
+    char *range_scratch = decode_in_ranges(desc) ? ws + w.total : nullptr;
+    return decode_impl(desc, qd, K, Z, Y, lse_dec, reinterpret_cast<uint32_t *>(workspace), st, range_scratch);
+}
+
+int flare_backward_variant(const flare_desc_t *desc, int shared_latents, const void *Q_enc, const void *Q_dec, const void *K,
+                           const void *V, const uint8_t *key_mask, const void *Y, const void *dY, const float *Z,
+                           const float *lse_enc, const float *lse_dec, float *dQ_enc, float *dQ_dec, void *dK, void *dV,
+                           void *workspace, size_t workspace_bytes, flare_stream_t stream) {
+    int rc = check_desc(desc);
+    if (rc != FLARE_OK) return rc;
+    const void *need[] = {Q_enc, K, V, Y, dY, Z, lse_enc, lse_dec, dQ_enc, dK, dV, workspace};
+    for (const void *p : need)
+        if (p == nullptr || !aligned16(p)) return FLARE_ERR_INVALID_ARG;
+    if ((Q_dec == nullptr) != (dQ_dec == nullptr)) return FLARE_ERR_INVALID_ARG;
+    if ((Q_dec && !aligned16(Q_dec)) || (dQ_dec && !aligned16(dQ_dec))) return FLARE_ERR_INVALID_ARG;
+    if ((rc = require_device()) != FLARE_OK) return rc;
+    const size_t base = flare_workspace_bytes(desc, FLARE_OP_BACKWARD);
+    const bool separate = Q_dec != nullptr;
+    const VariantLayout v = variant_layout(desc, FLARE_OP_BACKWARD, shared_latents, separate, base);
+    if (workspace_bytes < v.total) return FLARE_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = static_cast<char *>(workspace);
+    const int sms = device_info().sms;
+    const void *qe = Q_enc, *qd = Q_dec;
+    float *dqe = dQ_enc, *dqd = dQ_dec;
+    const long per = (long)desc->M * desc->D;
+    if (shared_latents) {
+        if ((rc = expand_heads(desc, Q_enc, ws + v.qe, st)) != FLARE_OK) return rc;
+        qe = ws + v.qe;
+        dqe = reinterpret_cast<float *>(ws + v.dq_full);
+        if (separate) {
+            if ((rc = expand_heads(desc, Q_dec, ws + v.qd, st)) != FLARE_OK) return rc;
+            qd = ws + v.qd;
+            dqd = reinterpret_cast<float *>(ws + v.dq2_full);
+        }
+    }
+    auto run = [&](const void *q, const float *le, const float *ld, float *dq, void *dk, bool skip_a) {
+        return desc->dtype == FLARE_DTYPE_F32
+                   ? backward_simt<float>(desc, sms, q, K, V, key_mask, Y, dY, Z, le, ld, dq, dk, dV, ws, st, skip_a)
+                   : backward_simt<__nv_bfloat16>(desc, sms, q, K, V, key_mask, Y, dY, Z, le, ld, dq, dk, dV, ws, st, skip_a);
+    };
+    if (!separate) {
+        if ((rc = run(qe, lse_enc, lse_dec, dqe, dK, false)) != FLARE_OK) return rc;
+    } else {
+        // Two runs of the backward over the same workspace.  With lse_enc = +inf every encode weight exp(S - lse_enc) is 0,
+        // so the first run (decode queries) leaves dZ, the decode term of dK and dQ_dec; with lse_dec = +inf the second
+        // (encode queries; dZ kept from the first) leaves the encode term of dK, dV and dQ_enc.
+        float *inf_enc = reinterpret_cast<float *>(ws + v.inf_enc), *inf_dec = reinterpret_cast<float *>(ws + v.inf_dec);
+        const long ne = (long)desc->B * desc->H * desc->M, nd = (long)desc->B * desc->N * desc->H;
+        fill_kernel<<<(unsigned)((ne + 255) / 256), 256, 0, st>>>(inf_enc, ne, INFINITY);
+        fill_kernel<<<(unsigned)((nd + 255) / 256), 256, 0, st>>>(inf_dec, nd, INFINITY);
+        FLARE_CUDA(cudaGetLastError());
+        void *dk2 = ws + v.dk2;
+        if ((rc = run(qd, inf_enc, lse_dec, dqd, dk2, false)) != FLARE_OK) return rc;
+        if ((rc = run(qe, lse_enc, inf_dec, dqe, dK, true)) != FLARE_OK) return rc;
+        const long nk = (long)desc->B * desc->N * desc->H * desc->D;
+        if (desc->dtype == FLARE_DTYPE_F32)
+            add_into_kernel<float><<<(unsigned)((nk + 255) / 256), 256, 0, st>>>((float *)dK, (const float *)dk2, nk);
+        else
+            add_into_kernel<__nv_bfloat16><<<(unsigned)((nk + 255) / 256), 256, 0, st>>>((__nv_bfloat16 *)dK, (const __nv_bfloat16 *)dk2, nk);
+        FLARE_CUDA(cudaGetLastError());
+    }
+    if (shared_latents) {
+        sum_heads_kernel<<<(unsigned)((per + 255) / 256), 256, 0, st>>>(dqe, dQ_enc, per, desc->H);
+        if (separate) sum_heads_kernel<<<(unsigned)((per + 255) / 256), 256, 0, st>>>(dqd, dQ_dec, per, desc->H);
+        FLARE_CUDA(cudaGetLastError());
+    }
     return FLARE_OK;
 }
 

@@ -52,6 +52,9 @@ _SIGNATURES = {
     "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 13 + [_sz, _vp]),
     "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
     "flare_check": (ctypes.c_int, [_vp, _vp]),
+    "flare_variant_workspace_bytes": (_sz, [_dp, ctypes.c_int, ctypes.c_int, ctypes.c_int]),
+    "flare_forward_variant": (ctypes.c_int, [_dp, ctypes.c_int] + [_vp] * 10 + [_sz, _vp]),
+    "flare_backward_variant": (ctypes.c_int, [_dp, ctypes.c_int] + [_vp] * 15 + [_sz, _vp]),
     "flare_spectral_gram": (ctypes.c_int, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "flare_spectral_eig": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int32, _vp, _vp, _vp, ctypes.c_int32, _vp]),
     "flare_launch_count": (ctypes.c_int, [_dp, ctypes.c_int]),
@@ -232,6 +235,37 @@ def flare_launch_count(desc: FlareDesc, op: int) -> int:
 
 def flare_selftest_wait(workspace, budget_ns: int, stream=None):
     _raise(load().flare_selftest_wait(_ptr(workspace, torch.uint8), int(budget_ns), _stream(stream)), "flare_selftest_wait")
+
+
+def flare_variant_workspace_bytes(desc, op, shared_latents, separate) -> int:
+    return int(load().flare_variant_workspace_bytes(ctypes.byref(desc), op, int(shared_latents), int(separate)))
+
+
+def flare_forward_variant(desc, shared_latents, Q_enc, Q_dec, K, V, key_mask, Y, Z, lse_enc, lse_dec, workspace, stream=None):
+    """The mixer with one latent sequence for all heads (Q [M, D]) and / or separate decode queries (Q_dec, else None)."""
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    qs = (M, D) if shared_latents else (H, M, D)
+    rc = load().flare_forward_variant(ctypes.byref(desc), int(shared_latents), _ptr(Q_enc, dt, qs), _ptr(Q_dec, dt, qs),
+                                      _ptr(K, dt, (B, N, H, D)), _ptr(V, dt, (B, N, H, D)), _ptr(key_mask, torch.uint8, (B, N)),
+                                      _ptr(Y, dt, (B, N, H, D)), _ptr(Z, torch.float32, (B, H, M, D)),
+                                      _ptr(lse_enc, torch.float32, (B, H, M)), _ptr(lse_dec, torch.float32, (B, N, H)),
+                                      _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
+    _raise(rc, "flare_forward_variant")
+
+
+def flare_backward_variant(desc, shared_latents, Q_enc, Q_dec, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ_enc, dQ_dec, dK,
+                           dV, workspace, stream=None):
+    dt = K.dtype
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    tok, qs = (B, N, H, D), ((M, D) if shared_latents else (H, M, D))
+    rc = load().flare_backward_variant(ctypes.byref(desc), int(shared_latents), _ptr(Q_enc, dt, qs), _ptr(Q_dec, dt, qs),
+                                       _ptr(K, dt, tok), _ptr(V, dt, tok), _ptr(key_mask, torch.uint8, (B, N)),
+                                       _ptr(Y, dt, tok), _ptr(dY, dt, tok), _ptr(Z, torch.float32, (B, H, M, D)),
+                                       _ptr(lse_enc, torch.float32, (B, H, M)), _ptr(lse_dec, torch.float32, (B, N, H)),
+                                       _ptr(dQ_enc, torch.float32, qs), _ptr(dQ_dec, torch.float32, qs), _ptr(dK, dt, tok),
+                                       _ptr(dV, dt, tok), _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
+    _raise(rc, "flare_backward_variant")
 
 
 def flare_spectral_gram(desc, Q, K, lse_enc, lse_dec, G, workspace, stream=None):

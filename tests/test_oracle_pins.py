@@ -263,6 +263,46 @@ def test_gram_of_algorithm_one_against_the_two_softmax_matrices(oracle):
         np.testing.assert_allclose(np.trace(G), np.sum(We * Wd.T), rtol=1e-12)
 
 
+def test_backward_with_separate_decode_queries(oracle):
+    """The asymmetric variant's gradients: against library autograd through two attention calls with different
+    queries (float64), against central differences in one entry of each query set, and, with Qd = Qe, against the
+    symmetric backward (dQe + dQd = dQ)."""
+    B, H, N, M, D = 2, 2, 19, 5, 4
+    inp = workloads.make_random(B, H, N, M, D, seed=53, with_dy=True, k_std=0.6)
+    Q, K, V, _, dY = _np(inp)
+    Qd = _np(workloads.make_random(B, H, N, M, D, seed=54))[0]
+    scale = 0.8
+    g = oracle.backward_asym(Q, Qd, K, V, dY, scale=scale)
+    Qe_t, Qd_t = torch.from_numpy(Q).requires_grad_(), torch.from_numpy(Qd).requires_grad_()
+    Kt, Vt = torch.from_numpy(K).requires_grad_(), torch.from_numpy(V).requires_grad_()
+    sdpa = torch.nn.functional.scaled_dot_product_attention
+    Kp, Vp = Kt.permute(0, 2, 1, 3), Vt.permute(0, 2, 1, 3)
+    Z = sdpa(Qe_t.unsqueeze(0).expand(B, -1, -1, -1), Kp, Vp, scale=scale)
+    Y = sdpa(Kp, Qd_t.unsqueeze(0).expand(B, -1, -1, -1), Z, scale=scale).permute(0, 2, 1, 3)
+    (Y * torch.from_numpy(dY)).sum().backward()
+    for name, t in (("dQe", Qe_t), ("dQd", Qd_t), ("dK", Kt), ("dV", Vt)):
+        np.testing.assert_allclose(g[name], t.grad.numpy(), rtol=1e-9, atol=1e-12, err_msg=name)
+
+    def loss(Qe_, Qd_):
+        Zl, _ = oracle.encode(Qe_, K, V, scale=scale)
+        Yl, _ = oracle.decode(Qd_, K, Zl, scale=scale)
+        return float((Yl * dY).sum())
+
+    eps = 1e-6
+    for which, idx in (("dQe", (1, 2, 3)), ("dQd", (0, 4, 1))):
+        Qp, Qm = (Q.copy(), Qd.copy()), (Q.copy(), Qd.copy())
+        k = 0 if which == "dQe" else 1
+        Qp[k][idx] += eps
+        Qm[k][idx] -= eps
+        fd = (loss(*Qp) - loss(*Qm)) / (2 * eps)
+        assert abs(fd - g[which][idx]) <= 1e-6 * max(1.0, abs(fd)), which
+    sym = oracle.backward(Q, K, V, dY, scale=scale)
+    same = oracle.backward_asym(Q, Q, K, V, dY, scale=scale)
+    np.testing.assert_allclose(same["dQe"] + same["dQd"], sym["dQ"], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(same["dK"], sym["dK"], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(same["dV"], sym["dV"], rtol=1e-11, atol=1e-13)
+
+
 def test_backward_rows_matches_full(oracle):
     """The sampled-rows backward is the full backward restricted to the listed tokens, bit for bit (dQ and dZ are
     full reductions in both)."""
