@@ -32,8 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) of one launch of each main kernel on the full mesh3d_1m workload, from the ncu captures
 # summarised under profiles/ (taken on a 262,144-token slice and scaled by 4: traffic is proportional to N).
 # Valid for the kernels as profiled; set to None when a kernel changes until the capture is redone.
-NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.330112e6 + 3.916544e6),
-               ("mesh3d_1m", "decode"): 4 * (68.004608e6 + 30.838016e6)}
+NCU_TRAFFIC = {("mesh3d_1m", "encode"): None, ("mesh3d_1m", "decode"): None}
 
 
 def get_workload(name: str) -> workloads.Workload:
@@ -144,6 +143,19 @@ def self_launch(n: int):
     raise SystemExit(subprocess.run(cmd).returncode)
 
 
+def run_micro():
+    """The instruction-level figures the kernels' design rests on, re-measured through flare_microbench."""
+    from paper_2508_12594_b200 import flare
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    names = ["exp_per_clk_per_sm_running_max_sfu", "exp_per_clk_per_sm_no_max_sfu", "exp_per_clk_per_sm_no_max_sfu_plus_fma",
+             "mma_unit_issue_cycles", "mma_commit_to_barrier_cycles"]
+    out = {}
+    for which, name in enumerate(names):
+        flare.flare_microbench(which, 2000 if which < 3 else 64)                      # warm-up
+        out[name] = flare.flare_microbench(which, 20000 if which < 3 else 256)
+    print(json.dumps({"micro": out}))
+
+
 def run_reference(args, w):
     """The reference arm: the oracle on the host cores, each step a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -182,6 +194,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override N (a smaller case of the same workload)")
     ap.add_argument("--no-backward", action="store_true", help="skip the forward+backward leg")
+    ap.add_argument("--micro", action="store_true", help="print the library's instruction-level measurements and exit")
     args = ap.parse_args()
     w = get_workload(args.workload)
     if args.tokens > 0:
@@ -190,6 +203,8 @@ def main():
         return self_launch(args.gpus)
     if args.impl == "reference":
         return run_reference(args, w)
+    if args.micro:
+        return run_micro()
     if args.warmup < 3:
         args.warmup = 3
 

@@ -21,7 +21,8 @@
  *     dQ_lat           [H, M, D]      float32    summed over the batch
  *
  * Padding (not in the paper): a masked token takes no part in the encode softmax; decode is evaluated for
- * every token.  A batch item with no valid token gets Z = 0, lse_enc = -inf.
+ * every token.  A batch item with no valid token gets Z = 0, lse_enc = -inf.  On the tensor-core path a masked
+ * token enters the products with weight exactly 0, so its rows of K and V must still hold finite numbers.
  *
  * Pointers and ownership: unless a function says "host", every pointer is a DEVICE pointer to memory owned
  * by the caller, 16-byte aligned; the library never allocates, frees or keeps them.  Calls enqueue work on
@@ -242,6 +243,19 @@ int flare_spectral_gram(const flare_desc_t *desc, const void *Q_lat, const void 
  */
 int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues, float *U, int32_t sweeps,
                        flare_stream_t stream);
+
+/*
+ * Instruction-level measurements behind the kernels' design (the paper has no counterpart), so that the figures the
+ * documentation quotes can be re-taken on the GPU at hand.  `which`:
+ *   0, 1, 2   exponentials per clock per SM of the softmax loop as the sixteen softmax warps of a forward kernel run it
+ *             (32 scores from tensor memory, 16 columns of packed weights back): 0 = with a running maximum and sum,
+ *             special-function unit only; 1 = without a maximum, special-function unit only; 2 = without a maximum,
+ *             every second pair of columns by the polynomial on the FMA pipe (what the fast forms run);
+ *   3, 4      cycles the issuing thread is held by one unit's tensor-core instructions (two value MMAs, one score MMA,
+ *             one commit), and cycles from the commit to the flip of its barrier.
+ * scratch: at least 4096 bytes of device memory.  *result is a HOST double.  Synchronises the stream.
+ */
+int flare_microbench(int which, int iters, void *scratch, size_t scratch_bytes, double *result, flare_stream_t stream);
 
 /*
  * After the stream has been synchronised: FLARE_OK, or FLARE_ERR_TIMEOUT if a kernel of the last call that

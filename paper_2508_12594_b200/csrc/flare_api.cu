@@ -14,6 +14,7 @@
 #include "flare_tc.cuh"
 #include "flare_bwd_tc.cuh"
 #include "flare_spectral.cuh"
+#include "flare_micro.cuh"
 
 using namespace flare;
 
@@ -124,7 +125,9 @@ bool use_tc(const flare_desc_t *d) {
         const char *e = std::getenv("FLARE_DEBUG_PATH");
         return e != nullptr && std::strcmp(e, "simt") == 0;
     }();
-    return !forced_simt && d->dtype == FLARE_DTYPE_BF16 && d->scale > 0.f &&
+    // (a scale so small that scale * kMaskedScore no longer dwarfs every real score would let padded tokens through the
+    // form that puts padding into the scores: such calls run on the CUDA cores too)
+    return !forced_simt && d->dtype == FLARE_DTYPE_BF16 && d->scale > 1e-20f &&
            (d->D == 16 || d->D == 32 || d->D == 64 || (d->D == 8 && d->H >= 2) || (d->D == 4 && d->H >= 4 && d->H % 2 == 0));
 }
 
@@ -1282,6 +1285,40 @@ int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues
     const size_t shmem = sizeof(float) * (4 * (size_t)pairs + M);
     spectral_jacobi_kernel<<<(unsigned)matrices, 256, shmem, (cudaStream_t)stream>>>(G, eigenvalues, U, M, sweeps);
     FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+int flare_microbench(int which, int iters, void *scratch, size_t scratch_bytes, double *result, flare_stream_t stream) {
+    if (!scratch || !result || !aligned16(scratch) || scratch_bytes < 4096 || which < 0 || which > 4) return FLARE_ERR_INVALID_ARG;
+    int rc = require_device();
+    if (rc != FLARE_OK) return rc;
+    if (iters < 1) iters = 1;
+    if (iters > 1000000) iters = 1000000;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int sms = device_info().sms > 512 ? 512 : device_info().sms;
+    unsigned long long *out = static_cast<unsigned long long *>(scratch);
+    FLARE_CUDA(cudaMemsetAsync(scratch, 0, 4096, st));
+    unsigned long long host[512];
+    if (which <= 2) {
+        if (which == 0) micro_softmax_kernel<0><<<sms, kTcThreads, 0, st>>>(iters, kLog2e, out);
+        if (which == 1) micro_softmax_kernel<1><<<sms, kTcThreads, 0, st>>>(iters, kLog2e, out);
+        if (which == 2) micro_softmax_kernel<2><<<sms, kTcThreads, 0, st>>>(iters, kLog2e, out);
+        FLARE_CUDA(cudaGetLastError());
+        FLARE_CUDA(cudaMemcpyAsync(host, out, sizeof(unsigned long long) * sms, cudaMemcpyDeviceToHost, st));
+        FLARE_CUDA(cudaStreamSynchronize(st));
+        double cycles = 0.0;
+        for (int i = 0; i < sms; ++i) cycles += (double)host[i];
+        cycles /= sms;
+        *result = cycles > 0.0 ? 512.0 * 32.0 * iters / cycles : 0.0;     // 512 threads x 32 columns per round
+    } else {
+        static std::atomic<uint64_t> smem_opt_in{0};
+        if (int rc_attr = ensure_big_smem(micro_mma_kernel, smem_opt_in, 64 * 1024)) return rc_attr;
+        micro_mma_kernel<<<1, 64, 24576 + 1024, st>>>(iters, out);
+        FLARE_CUDA(cudaGetLastError());
+        FLARE_CUDA(cudaMemcpyAsync(host, out, sizeof(unsigned long long) * 2, cudaMemcpyDeviceToHost, st));
+        FLARE_CUDA(cudaStreamSynchronize(st));
+        *result = (double)host[which - 3];
+    }
     return FLARE_OK;
 }
 

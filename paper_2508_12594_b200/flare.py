@@ -52,6 +52,7 @@ _SIGNATURES = {
     "flare_backward": (ctypes.c_int, [_dp] + [_vp] * 13 + [_sz, _vp]),
     "flare_forward_host": (ctypes.c_int, [_dp] + [_vp] * 11 + [_sz, _vp]),
     "flare_check": (ctypes.c_int, [_vp, _vp]),
+    "flare_microbench": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, _vp, _sz, ctypes.POINTER(ctypes.c_double), _vp]),
     "flare_variant_workspace_bytes": (_sz, [_dp, ctypes.c_int, ctypes.c_int, ctypes.c_int]),
     "flare_forward_variant": (ctypes.c_int, [_dp, ctypes.c_int] + [_vp] * 10 + [_sz, _vp]),
     "flare_backward_variant": (ctypes.c_int, [_dp, ctypes.c_int] + [_vp] * 15 + [_sz, _vp]),
@@ -266,6 +267,15 @@ def flare_backward_variant(desc, shared_latents, Q_enc, Q_dec, K, V, key_mask, Y
                                        _ptr(dQ_enc, torch.float32, qs), _ptr(dQ_dec, torch.float32, qs), _ptr(dK, dt, tok),
                                        _ptr(dV, dt, tok), _ptr(workspace, torch.uint8), workspace.numel(), _stream(stream))
     _raise(rc, "flare_backward_variant")
+
+
+def flare_microbench(which: int, iters: int = 20000, stream=None) -> float:
+    """One of the library's instruction-level measurements (see include/flare.h)."""
+    scratch = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    out = ctypes.c_double(0.0)
+    _raise(load().flare_microbench(int(which), int(iters), _ptr(scratch, torch.uint8), scratch.numel(), ctypes.byref(out),
+                                   _stream(stream)), "flare_microbench")
+    return float(out.value)
 
 
 def flare_spectral_gram(desc, Q, K, lse_enc, lse_dec, G, workspace, stream=None):

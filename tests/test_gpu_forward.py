@@ -263,3 +263,24 @@ def test_fast_forms_hand_over_only_when_out_of_range(oracle, k_std, redo):
     assert words[0] == 0 and bool(words[2]) == redo and bool(words[3]) == redo
     from tests._util import assert_stored_close
     assert_stored_close(to_np64(Y), oracle_forward(oracle, inp)["Y"], "bf16", f"fast forms, k_std={k_std}")
+
+
+def test_tiny_scale_keeps_padding_out(oracle):
+    """A scale so small that every score is practically zero, with a partial last tile: the tokens beyond N must still
+    get weight exactly 0 (the form of the encode kernel that marks padding by a huge negative score is not taken then)."""
+    inp = workloads.make_random(1, 2, 300, 256, 16, dtype="bf16", seed=13)
+    got, ref = gpu_forward(inp, scale=1e-24, canary=True), oracle_forward(oracle, inp, scale=1e-24)
+    assert_forward_close(got, ref, "bf16", "tiny scale")
+
+
+def test_microbenchmarks_are_in_range():
+    """The library's instruction-level measurements (the figures the kernel design quotes) on this GPU: the special-function
+    unit alone delivers about 15 exponentials per clock per SM in the softmax loop, half of them on the FMA pipe about 24;
+    a unit's tensor-core instructions hold the issuing thread for a few hundred cycles."""
+    sfu_max = flare.flare_microbench(0, 5000)
+    sfu = flare.flare_microbench(1, 5000)
+    both = flare.flare_microbench(2, 5000)
+    assert 11.0 <= sfu_max <= 16.5 and 11.0 <= sfu <= 16.5, (sfu_max, sfu)
+    assert 18.0 <= both <= 32.0 and both > 1.2 * sfu, (both, sfu)
+    issue, flip = flare.flare_microbench(3, 128), flare.flare_microbench(4, 128)
+    assert 100 <= issue <= 1200 and 50 <= flip <= 1200, (issue, flip)
