@@ -261,8 +261,7 @@ int flare_microbench(int which, int iters, void *scratch, size_t scratch_bytes, 
  * After the stream has been synchronised: FLARE_OK, or FLARE_ERR_TIMEOUT if a kernel of the last call that
  * used `workspace` gave up on a bounded wait (its outputs are then undefined).  Reads one word from the
  * workspace with a blocking copy.  workspace = NULL means the built-in scratch array of
- * flare_encode_static_scratch on the current device.  (flare_decode takes no workspace: a wait that gives up
- * there is not reported; use flare_forward, or the workspace of a following call, where that matters.)
+ * flare_encode_static_scratch on the current device.
  */
 int flare_check(const void *workspace, flare_stream_t stream);
 

@@ -270,7 +270,7 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast><<<grid, kFast ? kTcThreadsGuarded : kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
@@ -428,7 +428,7 @@ int launch_decode_stream_l(const flare_desc_t *d, int sms, const void *Q, const 
         const long four = (a.tiles + 3) / 4;                    // a CTA works on four tiles at a time
         if (per_head > four) per_head = four;
         if (per_head < 1) per_head = 1;
-        decode_stream_kernel<D, DRT, kPart, kM, kLse><<<dim3((unsigned)per_head, d->H, d->B), kTcThreads, smem, st>>>(tmK, tmQ, a);
+        decode_stream_kernel<D, DRT, kPart, kM, kLse><<<dim3((unsigned)per_head, d->H, d->B), kTcThreadsGuarded, smem, st>>>(tmK, tmQ, a);
         FLARE_CUDA(cudaGetLastError());
         return FLARE_OK;
     } else {

@@ -32,6 +32,11 @@ constexpr int kSoftmaxGroups = 4;                            // groups of 4 warp
 constexpr int kFirstIssuerWarp = 1;                          // warps 1..4: one MMA-issuing warp per group
 constexpr int kFirstSoftmaxWarp = kFirstIssuerWarp + kSoftmaxGroups;
 constexpr int kTcThreads = (kFirstSoftmaxWarp + 4 * kSoftmaxGroups) * 32;  // 672
+// The fast form of encode adds three guard warps behind the softmax warps (they check the norms of the key rows while a
+// tile waits in its stage; 24 warps still get 80 registers each: six per scheduler either way).
+constexpr int kGuardWarps = 3;
+constexpr int kFirstGuardWarp = kTcThreads / 32;
+constexpr int kTcThreadsGuarded = kTcThreads + 32 * kGuardWarps;          // 768
 constexpr int kTile = 128;       // tokens per tile (decode: TMEM lanes; encode: score columns)
 constexpr int kDecStages = 4;    // K tiles in flight (decode)
 constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode)
@@ -233,22 +238,26 @@ __device__ __forceinline__ void exp_chunk_fast(const uint32_t *r, uint32_t *pk, 
 }
 
 // Largest squared norm among the rows [lane, lane + 32, ...) < rows of a [rows, RB / 2] bf16 tile in shared memory
-// (the 16-byte chunks of a row are permuted by the swizzle, which a sum over the whole row does not see).
+// (the 16-byte chunks of a row are permuted by the swizzle, which a sum over the whole row does not see), as an upper
+// bound: the squares are summed two at a time in bf16 (one packed fma per pair of elements: the warp that runs this
+// shares its schedulers with the softmax warps, so instructions are what it costs), at most 16 roundings of 2^-9 per sum (3 %),
+// and the result is raised by 1/16 to stay above the exact value.
 template <int RB>
 __device__ __forceinline__ float tile_max_norm2(const uint8_t *tile, int rows, int lane) {
     float best = 0.f;
     for (int r = lane; r < rows; r += 32) {
-        float n2 = 0.f;
+        uint32_t acc0 = 0u, acc1 = 0u;                             // two bf16x2 sums
 #pragma unroll
         for (int c = 0; c < RB / 16; ++c) {
             const uint4 v = *reinterpret_cast<const uint4 *>(tile + (size_t)r * RB + c * 16);
-            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float a = __uint_as_float(u[k] << 16), b = __uint_as_float(u[k] & 0xffff0000u);
-                n2 = fmaf(a, a, fmaf(b, b, n2));
-            }
+            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc0) : "r"(v.x));
+            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc1) : "r"(v.y));
+            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc0) : "r"(v.z));
+            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc1) : "r"(v.w));
         }
+        float n2 = (__uint_as_float(acc0 << 16) + __uint_as_float(acc0 & 0xffff0000u)) +
+                   (__uint_as_float(acc1 << 16) + __uint_as_float(acc1 & 0xffff0000u));
+        n2 *= 1.0625f;
         if (!(n2 <= 3.0e38f)) n2 = INFINITY;                    // a row with a NaN or an infinity fails every check
         best = fmaxf(best, n2);
     }
@@ -751,7 +760,7 @@ struct DecodeStreamSmem {
 // matters most for the issuing thread (its scalar instructions wait for issue slots among the softmax warps).
 // kLse: the log-sum-exp rows are wanted (lse_dec; always with kPart): the threads then also add up the unrounded weights.
 template <int D, int DRT = 0, bool kPart = false, int kM = 0, bool kLse = false>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreadsGuarded, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, DecodeTcArgs a) {
     static_assert(D == 16 || D == 32, "head widths 16 (and narrower, as part of 16) and 32");
     constexpr bool kHalf = DRT != 0;
@@ -780,6 +789,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     constexpr int SUM_COL = 32;                                 // accumulator column of the row sum
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tid = threadIdx.x < kTcThreads ? (int)threadIdx.x : (1 << 30);   // the guard warps stage nothing
     const int h = blockIdx.y, b = blockIdx.z;
     const int off = kHalf ? narrow_offset(h, DR) : 0;
     const int t_begin = (int)((long)a.tiles * blockIdx.x / gridDim.x);
@@ -791,7 +801,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     if (threadIdx.x == 0) {
         for (int i = 0; i < NBARS; ++i) {
             const bool by_warps = (i >= P_FULL && i < P_FULL + 2 * NG) || (i >= Y_FREE && i < Y_FREE + NG);
-            ptx::mbar_init(bar(i), by_warps ? 4u : 1u);
+            const bool guarded = i >= K_EMPTY && i < K_EMPTY + kMaxStages;     // released by its group and its guard warp
+            ptx::mbar_init(bar(i), by_warps ? 4u : guarded ? 2u : 1u);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -802,7 +813,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     {   // Z_bh -> [hi | lo | ones] blocks of M latent-major rows in the swizzled layout of an MN-major B operand
         const float *Zg = a.Z + (((size_t)b * a.H + h) * a.mtot + a.m0) * DR;
         if (kHalf) {
-            for (int i = threadIdx.x; i < M * (D / 8); i += kTcThreads) {
+            for (int i = tid; i < M * (D / 8); i += kTcThreads) {
                 reinterpret_cast<uint4 *>(sQ)[i] = make_uint4(0, 0, 0, 0);
                 reinterpret_cast<uint4 *>(sZ)[i] = make_uint4(0, 0, 0, 0);
                 reinterpret_cast<uint4 *>(sZ + (size_t)M * G::RB)[i] = make_uint4(0, 0, 0, 0);
@@ -812,7 +823,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 stage_rows4<D>(sQ, a.Q + ((size_t)h * a.mtot + a.m0) * DR, M, off);
                 stage_rows4_hilo<D>(sZ, sZ + (size_t)M * G::RB, Zg, M, off);
             } else {
-                for (int i = threadIdx.x; i < M * (DR / 8); i += kTcThreads) {
+                for (int i = tid; i < M * (DR / 8); i += kTcThreads) {
                     const int m = i / (DR / 8), c = i % (DR / 8);
                     *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) =
                         *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * a.mtot + a.m0 + m) * DR + c * 8);
@@ -820,7 +831,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
         }
         constexpr int ZC = DR >= 8 ? DR / 8 : 1;
-        for (int i = threadIdx.x; i < (DR >= 8 ? M * ZC : 0); i += kTcThreads) {
+        for (int i = tid; i < (DR >= 8 ? M * ZC : 0); i += kTcThreads) {
             const int m = i / ZC, c = i % ZC;
             const float4 lo = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8);
             const float4 hi = *reinterpret_cast<const float4 *>(Zg + (size_t)m * DR + c * 8 + 4);
@@ -836,7 +847,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             *reinterpret_cast<uint4 *>(dst + (size_t)M * G::RB) = make_uint4(vl[0], vl[1], vl[2], vl[3]);
         }
         uint8_t *ones = sZ + (size_t)2 * M * G::RB;             // a one in column 0 of every latent row
-        for (int i = threadIdx.x; i < M * (G::RB / 16); i += kTcThreads) {
+        for (int i = tid; i < M * (G::RB / 16); i += kTcThreads) {
             const int m = i / (G::RB / 16), c = i % (G::RB / 16);
             *reinterpret_cast<uint4 *>(ones + (size_t)m * G::RB + ((c ^ G::swz(m)) << 4)) = make_uint4(c == 0 ? 0x00003F80u : 0u, 0, 0, 0);
         }
@@ -857,23 +868,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * a.mtot + a.m0 + r);
             }
         }
-        // The whole warp walks the tiles: lane 0 issues the loads; all lanes check the key rows of the tile a stage held
-        // before it is overwritten: |q| |k| sl2 <= kFastMaxLog2 for every latent row of the launch (whole rows: in
-        // the narrow forms they hold the neighbouring heads' features too, which only makes the check stricter).
-        bool tame = warp_wait(bar(Q_FULL), 0, abort_flag, kErrDecode | 9);
-        const float q2 = warp_max_nan(tile_max_norm2<G::RB>(sQ, M, lane));
-        const float lim = kFastMaxLog2 / a.sl2;
-        const float k2_limit = lim * lim / fmaxf(q2, 1e-30f);
-        if (!(q2 <= 3.0e38f)) tame = false;
-        auto check_tile = [&](int j) {
-            const int sj = j % nstages;
-            if (!warp_wait(bar(K_FULL + sj), (j / nstages) & 1, abort_flag, kErrDecode | 10)) return;
-            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sK + (size_t)sj * G::TILE_BYTES, kTile, lane));
-            if (!(k2 <= k2_limit)) tame = false;
-        };
         for (int i = 0; i < ntiles; ++i) {
             const int s = i % nstages;
-            if (i >= nstages) check_tile(i - nstages);
             if (!warp_wait(bar(K_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrDecode | 1)) break;
             if (lane == 0) {
                 ptx::mbar_arrive_expect_tx(bar(K_FULL + s), G::TILE_BYTES);
@@ -881,7 +877,23 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                                  (t_begin + i) * kTile, b);
             }
         }
-        for (int j = ntiles > nstages ? ntiles - nstages : 0; j < ntiles; ++j) check_tile(j);
+    } else if (warp >= kFirstGuardWarp) {
+        // Guard warps, one tile in three each: |q| |k| sl2 <= kFastMaxLog2 for every latent row of the launch and every
+        // key row of the tile, checked while the tile sits in its stage (whole rows: in the narrow forms they hold the
+        // neighbouring heads' features too, which only makes the check stricter).
+        bool tame = warp_wait(bar(Q_FULL), 0, abort_flag, kErrDecode | 9);
+        const float q2 = warp_max_nan(tile_max_norm2<G::RB>(sQ, M, lane));
+        const float lim = kFastMaxLog2 / a.sl2;
+        const float k2_limit = lim * lim / fmaxf(q2, 1e-30f);
+        if (!(q2 <= 3.0e38f)) tame = false;
+        for (int j = warp - kFirstGuardWarp; j < ntiles; j += kGuardWarps) {
+            const int sj = j % nstages;
+            if (!warp_wait(bar(K_FULL + sj), (j / nstages) & 1, abort_flag, kErrDecode | 10)) break;
+            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sK + (size_t)sj * G::TILE_BYTES, kTile, lane));
+            if (!(k2 <= k2_limit)) tame = false;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(K_EMPTY + sj));
+        }
         if (!tame && lane == 0 && a.redo != nullptr) *a.redo = 1u;
     } else if (warp < kFirstSoftmaxWarp) {
         const int g = warp - kFirstIssuerWarp;
@@ -1240,10 +1252,11 @@ constexpr float kDeadBelow = -1.0e29f;
 // which costs a bias tile and one more MMA per unit of the tiles that have padding, and nothing elsewhere.
 //
 // kFast: no running maximum (see kFastMaxLog2): weights 2^(s * sl2) as they stand, half of them by the polynomial
-// on the FMA pipe (not with kHiLo, whose point is accuracy), no rescaling, partial maximum 0.  The producer warp
-// checks the norms of the key rows of every tile it has loaded against those of the CTA's latent rows.
+// on the FMA pipe (not with kHiLo, whose point is accuracy), no rescaling, partial maximum 0.  Three more warps
+// (the guard warps) check the norms of the key rows of every tile against those of the CTA's latent rows; in the
+// producer warp that check sat between two loads and cost 10 % at D = 32 (measured).
 template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kFast ? kTcThreadsGuarded : kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
     static_assert(!(kFast && kDz), "the dZ form has no maximum to drop");
@@ -1268,6 +1281,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tid = threadIdx.x < kTcThreads ? (int)threadIdx.x : (1 << 30);   // the guard warps stage nothing
     const int M = a.M;
     // h: the head, or in the head-pair form the first head of the pair
     const int split = blockIdx.x, h = (kPair ? 2 : 1) * (blockIdx.y / a.pairs), pair = blockIdx.y % a.pairs, b = blockIdx.z;
@@ -1302,7 +1316,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
             ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? (kFast ? 4u : 128u)   // fast form: one arrival per warp
-                                   : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users
+                                   : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users + (kFast ? 1u : 0u)   // and its guard warp
                                    : (i >= KV_FULL && i < KV_FULL + kEncStages) ? 2u : 1u);   // the TMA loads, the bias tile
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -1312,19 +1326,19 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     if (warp == kFirstIssuerWarp) ptx::tmem_alloc(ptx::smem_u32(tmem_slot), NCOLS);
     // latent rows beyond M are zero so their (discarded) lanes stay finite
-    for (int i = threadIdx.x; i < (2 * kTile - rows_here) * (G::RB / 16); i += kTcThreads)
+    for (int i = tid; i < (2 * kTile - rows_here) * (G::RB / 16); i += kTcThreads)
         reinterpret_cast<uint4 *>(sQ + (size_t)rows_here * G::RB)[i] = make_uint4(0, 0, 0, 0);
     uint8_t *sBias = smem + SM::bias_off();                     // [stage] bias tiles, then the tile of ones
     if (!kDz) {
         using GB = TileGeom<16>;
         uint8_t *ones = sBias + (size_t)kEncStages * SM::kBiasTile;
-        for (int r = threadIdx.x; r < kTile; r += kTcThreads) {   // row r = [1, 0, ..., 0]: the first 16-byte chunk, swizzled
+        for (int r = tid; r < kTile; r += kTcThreads) {   // row r = [1, 0, ..., 0]: the first 16-byte chunk, swizzled
             reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r)] = make_uint4(0x00003F80u, 0, 0, 0);
             reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r) ^ 1] = make_uint4(0, 0, 0, 0);
         }
     }
     if (kOnes) {
-        for (int i = threadIdx.x; i < kTile * (G::RB / 16); i += kTcThreads) {
+        for (int i = tid; i < kTile * (G::RB / 16); i += kTcThreads) {
             const int r = i / (G::RB / 16), ch = i % (G::RB / 16);
             *reinterpret_cast<uint4 *>(sOnes + (size_t)r * G::RB + ((ch ^ G::swz(r)) << 4)) =
                 make_uint4(ch == 0 ? 0x00003F80u : 0u, 0, 0, 0);
@@ -1333,7 +1347,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (kPair) {
         // block-diagonal A operand: row r < 64 = [Q[h][r] | 0], row 64 + r = [0 | Q[h+1][r]], 16-byte chunks swizzled
         __syncthreads();
-        for (int i = threadIdx.x; i < 2 * M * (D / 8); i += kTcThreads) {
+        for (int i = tid; i < 2 * M * (D / 8); i += kTcThreads) {
             const int which = i / (M * (D / 8)), rem = i % (M * (D / 8)), m = rem / (D / 8), ch = rem % (D / 8);
             const uint4 v = *reinterpret_cast<const uint4 *>(a.Q + ((size_t)(h + which) * M + m) * D + ch * 8);
             const int r = which * 64 + m, chunk = which * (D / 8) + ch;
@@ -1346,7 +1360,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if constexpr (DR == 4) {
             stage_rows4<DG>(sQ, a.Q + ((size_t)h * M + lb0 * kTile) * DR, rows_q, off);
         } else {
-            for (int i = threadIdx.x; i < rows_q * (DR / 8); i += kTcThreads) {
+            for (int i = tid; i < rows_q * (DR / 8); i += kTcThreads) {
                 const int m = i / (DR / 8), ch = i % (DR / 8);
                 *reinterpret_cast<uint4 *>(sQ + (size_t)m * G::RB + ((ch ^ G::swz(m)) << 4)) =
                     *reinterpret_cast<const uint4 *>(a.Q + ((size_t)h * M + lb0 * kTile + m) * DR + ch * 8);
@@ -1369,29 +1383,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
             }
         }
-        // Fast form: the largest |k|^2 a tile may hold so that |q| |k| sl2 <= kFastMaxLog2 for the CTA's latent rows.
-        // (Whole rows of both operands: in the head-pair and narrow forms they hold the neighbouring heads' features
-        // too, which only makes the check stricter.)
-        float k2_limit = 0.f;
-        bool tame = true;
-        if (kFast) {
-            tame = warp_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 8);
-            const float q2 = warp_max_nan(tile_max_norm2<G::RB>(sQ, 2 * kTile, lane));
-            const float lim = kFastMaxLog2 / a.sl2;
-            k2_limit = lim * lim / fmaxf(q2, 1e-30f);
-            if (!(q2 <= 3.0e38f)) tame = false;                 // NaN or infinity in Q
-        }
-        auto check_tile = [&](int j) {                           // K tile j (relative to t_begin), still in its stage
-            const int sj = j % kEncStages;
-            if (!warp_wait(bar(KV_FULL + sj), (j / kEncStages) & 1, abort_flag, kErrEncode | 9)) return;
-            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sKV + (size_t)sj * 2 * G::TILE_BYTES, kTile, lane));
-            if (!(k2 <= k2_limit)) tame = false;
-        };
         // The whole warp walks the tiles: lane 0 waits for the stage and issues the loads; for a tile with padding
         // (masked tokens, or tokens beyond N) every lane first writes four rows of the stage's bias tile.
         for (int i = 0; i < nt; ++i) {
             const int s = i % kEncStages, t = t_begin + i;
-            if (kFast && i >= kEncStages) check_tile(i - kEncStages);   // the tile this stage held, before it is overwritten
             if (!warp_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
             const bool plain = kDz || kMaskBody || (a.key_mask == nullptr && (t + 1) * kTile <= a.N);
             if (!plain) {
@@ -1416,10 +1411,25 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ptx::tma_load_3d(ptx::smem_u32(dst + G::TILE_BYTES), &tmV, bar(KV_FULL + s), h * DR - off, t * kTile, b);
             }
         }
-        if (kFast) {
-            for (int j = nt > kEncStages ? nt - kEncStages : 0; j < nt; ++j) check_tile(j);   // the tiles still in their stages
-            if (!tame && lane == 0) *a.redo = 1u;
+    } else if (kFast && warp >= kFirstGuardWarp) {
+        // Guard warps (fast form), one tile in three each: the largest |k|^2 a tile may hold so that |q| |k| sl2 <=
+        // kFastMaxLog2 for the CTA's latent rows, checked while the tile sits in its stage; the stage is released by
+        // its users and its guard.  (Whole rows of both operands: in the head-pair and narrow forms they hold the
+        // neighbouring heads' features too, which only makes the check stricter.)
+        bool tame = warp_wait(bar(Q_FULL), 0, abort_flag, kErrEncode | 8);
+        const float q2 = warp_max_nan(tile_max_norm2<G::RB>(sQ, 2 * kTile, lane));
+        const float lim = kFastMaxLog2 / a.sl2;
+        const float k2_limit = lim * lim / fmaxf(q2, 1e-30f);
+        if (!(q2 <= 3.0e38f)) tame = false;                     // NaN or infinity in Q
+        for (int j = warp - kFirstGuardWarp; j < nt; j += kGuardWarps) {
+            const int sj = j % kEncStages;
+            if (!warp_wait(bar(KV_FULL + sj), (j / kEncStages) & 1, abort_flag, kErrEncode | 9)) break;
+            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sKV + (size_t)sj * 2 * G::TILE_BYTES, kTile, lane));
+            if (!(k2 <= k2_limit)) tame = false;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(KV_EMPTY + sj));
         }
+        if (!tame && lane == 0) *a.redo = 1u;
     } else if (warp < kFirstSoftmaxWarp) {
         const int g = warp - kFirstIssuerWarp;                  // the group this warp issues MMAs for
         const int j = g >> 1, c = g & 1;                        // its slot and column half
