@@ -137,14 +137,21 @@ std::atomic<int> g_path{FLARE_PATH_AUTO};
 // The fast forms (no running maximum, see kFastMaxLog2 in flare_tc.cuh) are followed by a launch of the exact
 // form that exits at once unless it is needed: two more launches per forward, which pay off from a few tens of
 // microseconds of work.
-bool use_fast(const flare_desc_t *d) {
+enum FastStage { kFastEncode, kFastDecode };
+bool use_fast(const flare_desc_t *d, FastStage stage) {
     if (!use_tc(d)) return false;
+    if (stage == kFastDecode && d->D > 32) return false;           // the streaming decode has no form for head width 64
     const int path = g_path.load(std::memory_order_relaxed);
     if (path == FLARE_PATH_EXACT) return false;
     if (path == FLARE_PATH_FAST) return true;
-    // (measured: below 256 latents a tile has too few units for the streaming forms to beat the exact ones, which
-    // hand a whole tile's row of scores over at once)
-    return d->M >= 256 && (double)d->B * d->H * d->N * d->M >= 3.0e7;
+    // Measured (forward stage times, fast against exact form): encode wins from 128 latents (3-5 % there, 15 % at 256),
+    // loses at 32 and 64 latents of width 32; the streaming decode
+    // wins from 64 latents (16 % at 64 and 128) and loses at 32; below some tens of microseconds of work the two extra
+    // launches cost more than the forms gain.
+    // (The head-pair form of encode, M <= 64, neither wins nor loses at D = 16 and loses at D = 32, where it has no room
+    // for the ones column and sums the weights in registers.)
+    const bool big_enough = d->M >= (stage == kFastEncode ? 128 : 64);
+    return big_enough && (double)d->B * d->H * d->N * d->M >= 3.0e7;
 }
 
 // Launch plan of the tensor-core encode: `pairs` CTAs per head along the latents (two 128-latent blocks each),
@@ -246,10 +253,11 @@ constexpr float kLog2e = 1.4426950408889634f;
 // outside the range it is valid for; the exact form that follows runs only then.
 constexpr int kRedoEncodeWord = 2, kRedoDecodeWord = 3;
 
-template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false>
-int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
-                     const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
-                     const float *lse_dec = nullptr, bool fallback = false) {
+// kAlt: one latent block (M <= 128), the CTA's two slots take alternate tiles: a form of its own with a deeper K/V ring
+template <int D, bool kPair, bool kDz, int DRT, bool kHiLo, bool kMaskBody, bool kFast, bool kAlt>
+int launch_encode_tc_a(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
+                       const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
+                       const float *lse_dec, bool fallback) {
     constexpr int DG = kPair ? 2 * D : D;
     CUtensorMap tmK, tmV, tmQ;
     int rc;
@@ -257,9 +265,9 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     if ((rc = make_token_map(&tmV, V, d, kTile, DG)) != FLARE_OK) return rc;
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
-    const size_t smem = EncodeSmem<DG>::total();
+    const size_t smem = EncodeSmem<DG, kAlt>::total();
     static std::atomic<uint64_t> smem_opt_in{0};
-    if (int rc_attr = ensure_big_smem(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast>, smem_opt_in, 227 * 1024)) return rc_attr;
+    if (int rc_attr = ensure_big_smem(encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast, kAlt>, smem_opt_in, 227 * 1024)) return rc_attr;
     EncodeTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.lse_dec = lse_dec;
@@ -270,13 +278,26 @@ int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q
     a.scale = d->scale; a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, (kPair ? d->H / 2 : d->H) * p.pairs, d->B);
-    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast><<<grid, kFast ? kTcThreadsGuarded : kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
+    encode_tc_kernel<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast, kAlt><<<grid, kFast ? kTcThreadsGuarded : kTcThreads, smem, st>>>(tmK, tmV, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }
 
-template <int D, int DRT, bool kPadded>
-int launch_bwd_dq_tc_p(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false>
+int launch_encode_tc(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V,
+                     const uint8_t *mask, float *pm, float *pl, float *pacc, uint32_t *status, cudaStream_t st,
+                     const float *lse_dec = nullptr, bool fallback = false) {
+    if constexpr (kPair) {
+        return launch_encode_tc_a<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st, lse_dec, fallback);
+    } else {
+        if (d->M <= kTile)
+            return launch_encode_tc_a<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast, true>(d, p, Q, K, V, mask, pm, pl, pacc, status, st, lse_dec, fallback);
+        return launch_encode_tc_a<D, kPair, kDz, DRT, kHiLo, kMaskBody, kFast, false>(d, p, Q, K, V, mask, pm, pl, pacc, status, st, lse_dec, fallback);
+    }
+}
+
+template <int D, int DRT, bool kPadded, bool kAlt>
+int launch_bwd_dq_tc_a(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
                      const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
                      const float *lse_dec, const float *dd, float *part, uint32_t *status, cudaStream_t st) {
     CUtensorMap tmK, tmV, tmG, tmQ;
@@ -286,9 +307,9 @@ int launch_bwd_dq_tc_p(const flare_desc_t *d, const TcEncodePlan &p, const void 
     if ((rc = make_token_map(&tmG, dY, d, kTile, D)) != FLARE_OK) return rc;
     if (DRT != 0) tmQ = tmK;   // unused: the narrow forms stage Q with their threads
     else if ((rc = make_latent_map(&tmQ, Q, d)) != FLARE_OK) return rc;
-    const size_t smem = BwdDqSmem<D>::total();
+    const size_t smem = BwdDqSmem<D, kAlt>::total();
     static std::atomic<uint64_t> smem_opt_in{0};
-    if (int rc_attr = ensure_big_smem(bwd_dq_tc_kernel<D, DRT, kPadded>, smem_opt_in, 227 * 1024)) return rc_attr;
+    if (int rc_attr = ensure_big_smem(bwd_dq_tc_kernel<D, DRT, kPadded, kAlt>, smem_opt_in, 227 * 1024)) return rc_attr;
     BwdDqTcArgs a;
     a.Q = static_cast<const __nv_bfloat16 *>(Q);
     a.Z = Z; a.dZ = dZ; a.lse_enc = lse_enc; a.de = de; a.lse_dec = lse_dec; a.dd = dd;
@@ -297,9 +318,19 @@ int launch_bwd_dq_tc_p(const flare_desc_t *d, const TcEncodePlan &p, const void 
     a.sl2 = d->scale * kLog2e;
     a.tiles = p.tiles; a.splits = p.splits; a.pairs = p.pairs; a.partials_per_split = p.per_split;
     dim3 grid(p.splits, d->H * p.pairs, d->B);
-    bwd_dq_tc_kernel<D, DRT, kPadded><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
+    bwd_dq_tc_kernel<D, DRT, kPadded, kAlt><<<grid, kTcThreads, smem, st>>>(tmK, tmV, tmG, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
+}
+
+// (one latent block, M <= 128: the form whose slots take alternate tiles, with a deeper tile ring)
+template <int D, int DRT, bool kPadded>
+int launch_bwd_dq_tc_p(const flare_desc_t *d, const TcEncodePlan &p, const void *Q, const void *K, const void *V, const void *dY,
+                     const uint8_t *mask, const float *Z, const float *dZ, const float *lse_enc, const float *de,
+                     const float *lse_dec, const float *dd, float *part, uint32_t *status, cudaStream_t st) {
+    if (d->M <= kTile)
+        return launch_bwd_dq_tc_a<D, DRT, kPadded, true>(d, p, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part, status, st);
+    return launch_bwd_dq_tc_a<D, DRT, kPadded, false>(d, p, Q, K, V, dY, mask, Z, dZ, lse_enc, de, lse_dec, dd, part, status, st);
 }
 
 template <int D, int DRT = 0>
@@ -735,7 +766,7 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
         TcEncodePlan p = tc_encode_plan(d, di.sms);
         uint32_t *status = reinterpret_cast<uint32_t *>(base);
         // a caller that asks for lse_enc is saving Z for the backward: weights as two bf16 halves (see exp_chunk_hilo)
-        const bool fast = use_fast(d);
+        const bool fast = use_fast(d, kFastEncode);
 #define FLARE_ENC3(DD, PAIR, DRT, MB, HL) encode_tc_forms<DD, PAIR, DRT, HL, MB>(d, p, Q, K, V, mask, pm, pl, pacc, status, st, fast)
 #define FLARE_ENC2(DD, PAIR, DRT, MB) (lse_enc != nullptr ? FLARE_ENC3(DD, PAIR, DRT, MB, true) : FLARE_ENC3(DD, PAIR, DRT, MB, false))
         // A call with a key mask has padding in every tile and takes the form that tests every element (see
@@ -788,7 +819,7 @@ size_t decode_range_bytes(const flare_desc_t *d) {
 template <int D, int DRT>
 int decode_tc_any(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *Z, void *Y, float *lse_dec,
                   uint32_t *status, char *range_scratch, cudaStream_t st) {
-    const bool fast = use_fast(d) && status != nullptr;
+    const bool fast = use_fast(d, kFastDecode) && status != nullptr;
     if (d->M <= kDecodeMaxM) return launch_decode_tc<D, DRT>(d, sms, Q, K, Z, Y, lse_dec, status, st, 0, 0, nullptr, fast);
     constexpr int DR = DRT ? DRT : D;
     const int C = decode_ranges(d);
@@ -849,8 +880,9 @@ int static_scratch_address(void **out) {
 
 // Kernels one call of `op` launches (the memset of the workspace header is not a kernel).
 int launches_for(const flare_desc_t *d, int op, int sms) {
-    const int f = use_fast(d) ? 2 : 1;                          // fast form, then the exact form (which may exit at once)
-    const int enc = f + 1;                                      // encode, merge
+    // a fast form is followed by the exact form (which may exit at once)
+    const int fe = use_fast(d, kFastEncode) ? 2 : 1, f = use_fast(d, kFastDecode) ? 2 : 1;
+    const int enc = fe + 1;                                     // encode, merge
     const int dec = decode_in_ranges(d) ? f * decode_ranges(d) + 1 : f;   // ranges of latents and their combination
     switch (op) {
         case FLARE_OP_ENCODE: return enc;

@@ -16,7 +16,8 @@
 
 namespace flare {
 
-constexpr int kBqStages = 3;     // (K, V, dY) tile triples in flight
+constexpr int kBqStages = 3;     // (K, V, dY) tile triples in flight where all four groups of a CTA work on the same tile
+constexpr int kBqMaxStages = 8;  // ... and at most where the two slots take alternate tiles (see kEncMaxStages)
 
 struct BwdDqTcArgs {
     const __nv_bfloat16 *Q;    // [H,M,D] (read directly in the half-width form)
@@ -32,15 +33,24 @@ struct BwdDqTcArgs {
     int tiles, splits, pairs, partials_per_split;
 };
 
-template <int D>
+template <int D, bool kAlt>
 struct BwdDqSmem {
     using G = TileGeom<D>;
+    static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 64 * sizeof(float);   // per softmax warp: 2 x 64 column constants
+    static constexpr size_t total_for(int n) {
+        return (size_t)n * 3 * G::TILE_BYTES + (size_t)5 * 2 * kTile * G::RB + 512 + kColBytes + 1024;
+    }
+    static constexpr int stages_for() {
+        int n = kAlt ? kBqMaxStages : kBqStages;
+        while (n > kBqStages && total_for(n) > 227 * 1024) --n;
+        return n;
+    }
+    static constexpr int kStages = stages_for();                 // (K, V, dY) tile triples in flight
     static constexpr size_t tile_off = 0;                        // [stage][K | V | dY]
-    __host__ __device__ static size_t q_off() { return (size_t)kBqStages * 3 * G::TILE_BYTES; }
+    __host__ __device__ static size_t q_off() { return (size_t)kStages * 3 * G::TILE_BYTES; }
     // Q, Z_hi, Z_lo, dZ_hi, dZ_lo: 256 latent rows each
     __host__ __device__ static size_t lat_off(int which) { return q_off() + (size_t)which * 2 * kTile * G::RB; }
     __host__ __device__ static size_t bar_off() { return lat_off(5); }
-    static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 64 * sizeof(float);   // per softmax warp: 2 x 64 column constants
     __host__ __device__ static size_t col_off() { return bar_off() + 512; }
     __host__ __device__ static size_t total() {
         size_t t = col_off() + kColBytes + 1024;
@@ -52,13 +62,15 @@ struct BwdDqSmem {
 // kernels (the head is DRT wide in memory; token tiles carry the neighbouring heads' features beside the head's
 // own, every latent operand zeros there, and the other columns of the partial dQ are dropped).
 // kPadded: the launch has padded tokens (a key mask, or N not a multiple of the tile); without it the unit body that
-// tests validity is not compiled in.
-template <int D, int DRT = 0, bool kPadded = true>
+// tests validity is not compiled in.  kAlt: one latent block (the host picks this form for M <= 128), the two slots take
+// alternate tiles and the tile ring is as deep as fits.
+template <int D, int DRT = 0, bool kPadded = true, bool kAlt = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmQ, BwdDqTcArgs a) {
     using G = TileGeom<D>;
-    using SM = BwdDqSmem<D>;
+    using SM = BwdDqSmem<D, kAlt>;
+    constexpr int nstages = SM::kStages;                        // depth of the tile ring
     constexpr bool kHalf = DRT != 0;
     constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     extern __shared__ uint8_t smem_raw[];
@@ -68,7 +80,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off());
     constexpr int NG = kSoftmaxGroups;
     // per group: S_FULL and P_FULL for each of its two unit buffers
-    enum { T_FULL = 0, T_EMPTY = T_FULL + kBqStages, S_FULL = T_EMPTY + kBqStages, P_FULL = S_FULL + 2 * NG,
+    enum { T_FULL = 0, T_EMPTY = T_FULL + nstages, S_FULL = T_EMPTY + nstages, P_FULL = S_FULL + 2 * NG,
            ACC_DONE = P_FULL + 2 * NG, Q_FULL = ACC_DONE + NG, NBARS };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
@@ -80,7 +92,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int t_end = (int)((long)a.tiles * (split + 1) / a.splits);
     const int nt = t_end - t_begin;
     const int MB = (M + kTile - 1) / kTile;
-    const bool alternate = (MB == 1);                           // one latent block: the two slots take alternate tiles
+    const bool alternate = kAlt || MB == 1;                           // one latent block: the two slots take alternate tiles
     const int lb0 = pair * 2;
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
@@ -94,7 +106,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
             ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? 128u
-                                   : (i >= T_EMPTY && i < T_EMPTY + kBqStages) ? users : 1u);
+                                   : (i >= T_EMPTY && i < T_EMPTY + nstages) ? users : 1u);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
@@ -157,8 +169,8 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ptx::tma_load_2d(ptx::smem_u32(sQ + (size_t)r * G::RB), &tmQ, bar(Q_FULL), 0, h * M + lb0 * kTile + r);
             }
             for (int i = 0; i < nt; ++i) {
-                const int s = i % kBqStages;
-                if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / kBqStages) & 1) ^ 1, abort_flag, kErrBwdDq | 1)) break;
+                const int s = i % nstages;
+                if (!ptx::mbar_wait(bar(T_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrBwdDq | 1)) break;
                 ptx::mbar_arrive_expect_tx(bar(T_FULL + s), 3 * G::TILE_BYTES);
                 uint8_t *dst = sT + (size_t)s * 3 * G::TILE_BYTES;
                 ptx::tma_load_3d(ptx::smem_u32(dst), &tmK, bar(T_FULL + s), h * DR - off, (t_begin + i) * kTile, b);
@@ -186,8 +198,8 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             int t_s = alternate ? j : 0, t_v = t_s;                         // tiles of the next tile-unit / dQ-unit
             const int t_step = alternate ? 2 : 1;
             auto issue_tiles = [&](int n) -> bool {
-                const int s = t_s % kBqStages, w = n % UPH;
-                if (w == 0 && !ptx::mbar_wait(bar(T_FULL + s), (t_s / kBqStages) & 1, abort_flag, kErrBwdDq | 3)) return false;
+                const int s = t_s % nstages, w = n % UPH;
+                if (w == 0 && !ptx::mbar_wait(bar(T_FULL + s), (t_s / nstages) & 1, abort_flag, kErrBwdDq | 3)) return false;
                 ptx::tc_fence_after();
                 const uint32_t tbase = ptx::smem_u32(sT + (size_t)s * 3 * G::TILE_BYTES);
                 const uint64_t rowoff = (uint64_t)((c * HALF + w * UNIT) * G::RB / 16);   // the unit's 16 token rows
@@ -212,7 +224,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             };
             for (int n = 0; ok && n < 2 && n < units; ++n) ok = issue_tiles(n);
             for (int n = 0; ok && n < units; ++n) {
-                const int s = t_v % kBqStages, w = n % UPH;
+                const int s = t_v % nstages, w = n % UPH;
                 if (!ptx::mbar_wait(bar(P_FULL + 2 * g + (n & 1)), (n >> 1) & 1, abort_flag, kErrBwdDq | 4)) { ok = false; break; }
                 ptx::tc_fence_after();
                 // dQ_part += dS_unit K_unit (hi, then lo half of dS): the unit's 16 token rows of the K tile as the

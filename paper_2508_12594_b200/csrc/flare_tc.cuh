@@ -38,8 +38,12 @@ constexpr int kGuardWarps = 3;
 constexpr int kFirstGuardWarp = kTcThreads / 32;
 constexpr int kTcThreadsGuarded = kTcThreads + 32 * kGuardWarps;          // 768
 constexpr int kTile = 128;       // tokens per tile (decode: TMEM lanes; encode: score columns)
-constexpr int kDecStages = 4;    // K tiles in flight (decode)
-constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode)
+constexpr int kDecStages = 4;    // K tiles in flight (decode); 8 and 12 were measured 10 % slower at 32 and 128 latents
+constexpr int kEncStages = 3;    // K+V tile pairs in flight (encode), where all four groups of a CTA work on the same tile
+// Where the CTA's two slots take alternate tiles (one latent block: M <= 128) four tiles are in use at any time (per
+// slot the one whose weights are being formed and the next, whose scores are issued ahead) and a tile lasts half as
+// long, so the ring is as deep as shared memory allows: with three stages every load's latency was exposed (measured).
+constexpr int kEncMaxStages = 8;
 constexpr size_t kTcMinSmem = 120 * 1024;  // request at least this much so that one CTA owns an SM (and its TMEM)
 
 // Error codes left in the workspace header by a wait that gave up.
@@ -242,21 +246,41 @@ __device__ __forceinline__ void exp_chunk_fast(const uint32_t *r, uint32_t *pk, 
 // bound: the squares are summed two at a time in bf16 (one packed fma per pair of elements: the warp that runs this
 // shares its schedulers with the softmax warps, so instructions are what it costs), at most 16 roundings of 2^-9 per sum (3 %),
 // and the result is raised by 1/16 to stay above the exact value.
-template <int RB>
+// kHalves = 2 (head-pair form: a row holds two heads side by side): the larger of the two halves' sums, since a score
+// only ever meets one head's features.
+template <int RB, int kHalves = 1>
 __device__ __forceinline__ float tile_max_norm2(const uint8_t *tile, int rows, int lane) {
+    using G = TileGeom<RB / 2>;
     float best = 0.f;
     for (int r = lane; r < rows; r += 32) {
-        uint32_t acc0 = 0u, acc1 = 0u;                             // two bf16x2 sums
+        float n2;
+        if (kHalves == 1) {
+            uint32_t acc0 = 0u, acc1 = 0u;                         // two bf16x2 sums
 #pragma unroll
-        for (int c = 0; c < RB / 16; ++c) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(tile + (size_t)r * RB + c * 16);
-            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc0) : "r"(v.x));
-            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc1) : "r"(v.y));
-            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc0) : "r"(v.z));
-            asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc1) : "r"(v.w));
+            for (int c = 0; c < RB / 16; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(tile + (size_t)r * RB + c * 16);
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc0) : "r"(v.x));
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc1) : "r"(v.y));
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc0) : "r"(v.z));
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(acc1) : "r"(v.w));
+            }
+            n2 = (__uint_as_float(acc0 << 16) + __uint_as_float(acc0 & 0xffff0000u)) +
+                 (__uint_as_float(acc1 << 16) + __uint_as_float(acc1 & 0xffff0000u));
+        } else {
+            uint32_t acc[2] = {0u, 0u};                            // one bf16x2 sum per half of the row
+            const int sw = G::swz(r);
+#pragma unroll
+            for (int l = 0; l < RB / 16; ++l) {                    // logical chunk l sits at chunk l ^ swz(r)
+                const uint4 v = *reinterpret_cast<const uint4 *>(tile + (size_t)r * RB + ((l ^ sw) << 4));
+                uint32_t &a = acc[l >= RB / 32 ? 1 : 0];
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(a) : "r"(v.x));
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(a) : "r"(v.y));
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(a) : "r"(v.z));
+                asm("fma.rn.bf16x2 %0, %1, %1, %0;" : "+r"(a) : "r"(v.w));
+            }
+            n2 = fmaxf(__uint_as_float(acc[0] << 16) + __uint_as_float(acc[0] & 0xffff0000u),
+                       __uint_as_float(acc[1] << 16) + __uint_as_float(acc[1] & 0xffff0000u));
         }
-        float n2 = (__uint_as_float(acc0 << 16) + __uint_as_float(acc0 & 0xffff0000u)) +
-                   (__uint_as_float(acc1 << 16) + __uint_as_float(acc1 & 0xffff0000u));
         n2 *= 1.0625f;
         if (!(n2 <= 3.0e38f)) n2 = INFINITY;                    // a row with a NaN or an infinity fails every check
         best = fmaxf(best, n2);
@@ -1193,20 +1217,33 @@ struct EncodeTcArgs {
     int partials_per_split;  // 4 when M <= 128 (two slots alternate tiles, two column halves each), else 2
 };
 
-// DG: columns of a K/V tile row as the kernel sees it (D, or 2D in the head-pair form).
-template <int DG>
+// DG: columns of a K/V tile row as the kernel sees it (D, or 2D in the head-pair form).  kAlt: the CTA's two slots
+// take alternate tiles (one latent block); the ring is then as deep as fits, at most kEncMaxStages.
+template <int DG, bool kAlt>
 struct EncodeSmem {
     using G = TileGeom<DG>;
-    static constexpr size_t kv_off = 0;                         // [stage][K tile | V tile]
-    __host__ __device__ static size_t q_off() { return (size_t)kEncStages * 2 * G::TILE_BYTES; }
-    __host__ __device__ static size_t bar_off() { return q_off() + (size_t)2 * kTile * G::RB; }
     static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 32 * sizeof(float);   // per softmax warp: 2 x 32 column addends
-    __host__ __device__ static size_t col_off() { return bar_off() + 512; }
     // score bias of padded tokens: per stage a [128 tokens, 16] bf16 tile, then one [128 latents, 16] tile of ones
     static constexpr size_t kBiasTile = kTile * 32;
+    static constexpr size_t total_for(int n) {
+        size_t t = (size_t)n * 2 * G::TILE_BYTES + (size_t)2 * kTile * G::RB + 512 + kColBytes;
+        t = (t + 1023) & ~(size_t)1023;
+        t = (t + (size_t)(n + 1) * kBiasTile + 1023) & ~(size_t)1023;
+        return t + (size_t)kTile * G::RB + 1024;
+    }
+    static constexpr int stages_for() {
+        int n = kAlt ? kEncMaxStages : kEncStages;
+        while (n > kEncStages && total_for(n) > 227 * 1024) --n;
+        return n;
+    }
+    static constexpr int kStages = stages_for();                // K+V tile pairs in flight
+    static constexpr size_t kv_off = 0;                         // [stage][K tile | V tile]
+    __host__ __device__ static size_t q_off() { return (size_t)kStages * 2 * G::TILE_BYTES; }
+    __host__ __device__ static size_t bar_off() { return q_off() + (size_t)2 * kTile * G::RB; }
+    __host__ __device__ static size_t col_off() { return bar_off() + 512; }
     __host__ __device__ static size_t bias_off() { return (col_off() + kColBytes + 1023) & ~(size_t)1023; }
     // fast form: a [128 tokens, DG] tile with a one in column 0 of every row, the value operand's second block along N
-    __host__ __device__ static size_t ones_off() { return (bias_off() + (kEncStages + 1) * kBiasTile + 1023) & ~(size_t)1023; }
+    __host__ __device__ static size_t ones_off() { return (bias_off() + (kStages + 1) * kBiasTile + 1023) & ~(size_t)1023; }
     __host__ __device__ static size_t total() {
         size_t t = ones_off() + (size_t)kTile * G::RB + 1024;
         return t < kTcMinSmem ? kTcMinSmem : t;
@@ -1255,7 +1292,7 @@ constexpr float kDeadBelow = -1.0e29f;
 // on the FMA pipe (not with kHiLo, whose point is accuracy), no rescaling, partial maximum 0.  Three more warps
 // (the guard warps) check the norms of the key rows of every tile against those of the CTA's latent rows; in the
 // producer warp that check sat between two loads and cost 10 % at D = 32 (measured).
-template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false>
+template <int D, bool kPair, bool kDz = false, int DRT = 0, bool kHiLo = false, bool kMaskBody = false, bool kFast = false, bool kAlt = kPair>
 __global__ void __launch_bounds__(kFast ? kTcThreadsGuarded : kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, EncodeTcArgs a) {
@@ -1266,7 +1303,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     constexpr int DG = kPair ? 2 * D : D;
     constexpr int DR = kHalf ? DRT : D;                         // head width in memory
     using G = TileGeom<DG>;
-    using SM = EncodeSmem<DG>;
+    using SM = EncodeSmem<DG, kAlt>;
+    static_assert(kAlt || !kPair, "head pairs share one latent block");
+    constexpr int nstages = SM::kStages;                        // depth of the K/V ring
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *sKV = smem + SM::kv_off;
@@ -1274,7 +1313,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off());
     constexpr int NG = kSoftmaxGroups;
     // per group: S_FULL and P_FULL for each of its two score buffers, PV_DONE (one phase per unit), ACC_DONE
-    enum { KV_FULL = 0, KV_EMPTY = KV_FULL + kEncStages, S_FULL = KV_EMPTY + kEncStages, P_FULL = S_FULL + 2 * NG,
+    enum { KV_FULL = 0, KV_EMPTY = KV_FULL + nstages, S_FULL = KV_EMPTY + nstages, P_FULL = S_FULL + 2 * NG,
            PV_DONE = P_FULL + 2 * NG, ACC_DONE = PV_DONE + NG, Q_FULL = ACC_DONE + NG, NBARS };
     static_assert(NBARS * 8 + 8 <= 512, "barrier area too small");
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
@@ -1290,7 +1329,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int nt = t_end - t_begin;
     const int MB = (M + kTile - 1) / kTile;
     // job q -> (tile, slot); see the kernel comment
-    const bool alternate = (MB == 1);
+    // (the host picks the kAlt form for MB == 1; kept a run-time value in the other form, where it is always false: as
+    // a compile-time constant the same kernel measured 3 % slower, 0.613 against 0.592 ms on the million-point shape)
+    const bool alternate = kAlt || MB == 1;
     const int lb0 = pair * 2;                                   // latent block of slot 0
     const int nslots = alternate ? 2 : ((lb0 + 1 < MB) ? 2 : 1);
     const int nq = alternate ? nt : nt * nslots;
@@ -1316,8 +1357,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const uint32_t users = alternate ? 2u : 2u * (uint32_t)nslots;
         for (int i = 0; i < NBARS; ++i)
             ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + 2 * NG) ? (kFast ? 4u : 128u)   // fast form: one arrival per warp
-                                   : (i >= KV_EMPTY && i < KV_EMPTY + kEncStages) ? users + (kFast ? 1u : 0u)   // and its guard warp
-                                   : (i >= KV_FULL && i < KV_FULL + kEncStages) ? 2u : 1u);   // the TMA loads, the bias tile
+                                   : (i >= KV_EMPTY && i < KV_EMPTY + nstages) ? users + (kFast ? 1u : 0u)   // and its guard warp
+                                   : (i >= KV_FULL && i < KV_FULL + nstages) ? 2u : 1u);   // the TMA loads, the bias tile
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
@@ -1331,7 +1372,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint8_t *sBias = smem + SM::bias_off();                     // [stage] bias tiles, then the tile of ones
     if (!kDz) {
         using GB = TileGeom<16>;
-        uint8_t *ones = sBias + (size_t)kEncStages * SM::kBiasTile;
+        uint8_t *ones = sBias + (size_t)nstages * SM::kBiasTile;
         for (int r = tid; r < kTile; r += kTcThreads) {   // row r = [1, 0, ..., 0]: the first 16-byte chunk, swizzled
             reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r)] = make_uint4(0x00003F80u, 0, 0, 0);
             reinterpret_cast<uint4 *>(ones + (size_t)r * GB::RB)[GB::swz(r) ^ 1] = make_uint4(0, 0, 0, 0);
@@ -1386,8 +1427,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // The whole warp walks the tiles: lane 0 waits for the stage and issues the loads; for a tile with padding
         // (masked tokens, or tokens beyond N) every lane first writes four rows of the stage's bias tile.
         for (int i = 0; i < nt; ++i) {
-            const int s = i % kEncStages, t = t_begin + i;
-            if (!warp_wait(bar(KV_EMPTY + s), ((i / kEncStages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
+            const int s = i % nstages, t = t_begin + i;
+            if (!warp_wait(bar(KV_EMPTY + s), ((i / nstages) & 1) ^ 1, abort_flag, kErrEncode | 1)) break;
             const bool plain = kDz || kMaskBody || (a.key_mask == nullptr && (t + 1) * kTile <= a.N);
             if (!plain) {
                 using GB = TileGeom<16>;
@@ -1422,9 +1463,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const float k2_limit = lim * lim / fmaxf(q2, 1e-30f);
         if (!(q2 <= 3.0e38f)) tame = false;                     // NaN or infinity in Q
         for (int j = warp - kFirstGuardWarp; j < nt; j += kGuardWarps) {
-            const int sj = j % kEncStages;
-            if (!warp_wait(bar(KV_FULL + sj), (j / kEncStages) & 1, abort_flag, kErrEncode | 9)) break;
-            const float k2 = warp_max_nan(tile_max_norm2<G::RB>(sKV + (size_t)sj * 2 * G::TILE_BYTES, kTile, lane));
+            const int sj = j % nstages;
+            if (!warp_wait(bar(KV_FULL + sj), (j / nstages) & 1, abort_flag, kErrEncode | 9)) break;
+            const float k2 = warp_max_nan(tile_max_norm2<G::RB, kPair ? 2 : 1>(sKV + (size_t)sj * 2 * G::TILE_BYTES, kTile, lane));
             if (!(k2 <= k2_limit)) tame = false;
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(KV_EMPTY + sj));
@@ -1466,14 +1507,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const uint32_t sfull = bar(S_FULL + 2 * g), pfull = bar(P_FULL + 2 * g);
                 // without kMaskBody only a last partial tile has padding; its scores get the bias MMA (see kMaskedScore)
                 const int bias_tile = (!kMaskBody && a.N % kTile != 0) ? a.tiles - 1 - t_begin : -1;
-                int ss = t_s % kEncStages, sp = (t_s / kEncStages) & 1, sv = ss;
+                int ss = t_s % nstages, sp = (t_s / nstages) & 1, sv = ss;
                 auto scores = [&](int w) {                        // the scores of unit w of the S stream's tile, and the commit
                     const uint64_t kd = kd0 + (uint64_t)(stage_step * (uint32_t)ss + unit_step * (uint32_t)w);
 #pragma unroll
                     for (int k = 0; k < DG / 16; ++k) ptx::mma_ss(gcol + w * UNIT, qdesc + 2 * k, kd + 2 * k, idescS, k > 0);
                     if (!kMaskBody && t_s == bias_tile) {
                         using GB = TileGeom<16>;
-                        const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)kEncStages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
+                        const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)nstages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
                         const uint64_t bdesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)ss * SM::kBiasTile), 16, GB::SBO, GB::SWZ) +
                                                (uint64_t)((c * HALF + w * UNIT) * GB::RB / 16);
                         ptx::mma_ss(gcol + w * UNIT, odesc, bdesc, idescS, 1u);
@@ -1488,7 +1529,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 auto next_s = [&]() {
                     t_s += t_step;
                     ss += t_step;
-                    if (ss >= kEncStages) { ss -= kEncStages; sp ^= 1; }
+                    if (ss >= nstages) { ss -= nstages; sp ^= 1; }
                 };
                 if (ok && jobs > 0 && (ok = open_tile())) {
                     scores(0);
@@ -1509,7 +1550,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         if (w == 1) {                             // the tile's last unit: one arrival per group
                             ptx::mma_commit(bar(KV_EMPTY + sv));
                             sv += t_step;
-                            if (sv >= kEncStages) sv -= kEncStages;
+                            if (sv >= nstages) sv -= nstages;
                         }
                         if (job + 1 < jobs) {                     // the same unit of the group's next tile, into the buffer just read
                             if (w == 0 && !open_tile()) { ok = false; break; }
@@ -1520,7 +1561,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 if (ok) ptx::mma_commit(bar(ACC_DONE + g));
             } else {
-                int s_stage = t_s % kEncStages, s_phase = (t_s / kEncStages) & 1;   // stage and phase of the S stream's tile
+                int s_stage = t_s % nstages, s_phase = (t_s / nstages) & 1;   // stage and phase of the S stream's tile
                 auto issue_scores = [&](int n) -> bool {
                     const int s = s_stage, w = n & 1;                        // w: which 32 tokens of the half; also the buffer
                     if (!ptx::mbar_wait(bar(KV_FULL + s), s_phase, abort_flag, kErrEncode | 3)) return false;
@@ -1534,7 +1575,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (!kDz && !kMaskBody && !(a.key_mask == nullptr && (tile + 1) * kTile <= a.N)) {
                         // scores += ones x bias: padded tokens drop to kMaskedScore (see there)
                         using GB = TileGeom<16>;
-                        const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)kEncStages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
+                        const uint64_t odesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)nstages * SM::kBiasTile), 16, GB::SBO, GB::SWZ);
                         const uint64_t bdesc = ptx::smem_desc(ptx::smem_u32(sBias + (size_t)s * SM::kBiasTile), 16, GB::SBO, GB::SWZ) +
                                                (uint64_t)((c * HALF + w * UNIT) * GB::RB / 16);
                         ptx::mma_ss(gcol + w * UNIT, odesc, bdesc, idescS, 1u);
@@ -1543,12 +1584,12 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (w == 1) {
                         t_s += t_step;
                         s_stage += t_step;
-                        if (s_stage >= kEncStages) { s_stage -= kEncStages; s_phase ^= 1; }
+                        if (s_stage >= nstages) { s_stage -= nstages; s_phase ^= 1; }
                     }
                     return true;
                 };
                 for (int n = 0; ok && n < 2 && n < units; ++n) ok = issue_scores(n);
-                int v_stage = t_v % kEncStages;
+                int v_stage = t_v % nstages;
                 for (int n = 0; ok && n < units; ++n) {
                     const int w = n & 1, s = v_stage;
                     if (!ptx::mbar_wait(bar(P_FULL + 2 * g + w), (n >> 1) & 1, abort_flag, kErrEncode | 4)) break;
@@ -1567,7 +1608,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ptx::mma_commit(bar(KV_EMPTY + s));
                         t_v += t_step;
                         v_stage += t_step;
-                        if (v_stage >= kEncStages) v_stage -= kEncStages;
+                        if (v_stage >= nstages) v_stage -= nstages;
                     }
                     if (n + 2 < units) ok = issue_scores(n + 2);
                 }
