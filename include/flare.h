@@ -33,7 +33,9 @@
  * Supported shapes: D in {4, 8, 16, 32, 64}; float32: any M >= 1; bfloat16: M a multiple of 16, 16 <= M <= 2048.
  * bfloat16 inputs are multiplied on the tensor cores with float32 accumulation (D = 8 and 4 as part of a 16-wide
  * product whose other columns meet zeros; tensors of fewer than 16 feature columns, or with D = 4 and an odd
- * number of heads, on the CUDA cores).
+ * number of heads, on the CUDA cores).  float16 inputs (the type the paper trains in under autocast; any M >= 1) are
+ * accepted by every entry point and run on the CUDA-core kernels with float32 arithmetic: the tensor-core kernels are
+ * written for bfloat16 operands, whose wider exponent the forms without a running maximum rely on.
  *
  * Every entry point returns a flare_status_t; nothing is thrown, nothing is printed.
  */
@@ -59,7 +61,7 @@ typedef enum {
     FLARE_ERR_TIMEOUT = 6              /* a bounded device-side wait gave up (reported by flare_check) */
 } flare_status_t;
 
-enum { FLARE_DTYPE_F32 = 0, FLARE_DTYPE_BF16 = 1 };
+enum { FLARE_DTYPE_F32 = 0, FLARE_DTYPE_BF16 = 1, FLARE_DTYPE_F16 = 2 };
 enum { FLARE_OP_ENCODE = 0, FLARE_OP_DECODE = 1, FLARE_OP_FORWARD = 2, FLARE_OP_BACKWARD = 3, FLARE_OP_SPECTRAL = 4 };
 
 typedef struct {

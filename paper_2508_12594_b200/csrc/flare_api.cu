@@ -87,7 +87,7 @@ int check_desc(const flare_desc_t *d) {
     if (d == nullptr) return FLARE_ERR_INVALID_ARG;
     if (d->B <= 0 || d->H <= 0 || d->N <= 0 || d->M <= 0 || d->D <= 0) return FLARE_ERR_INVALID_ARG;
     if (!std::isfinite(d->scale)) return FLARE_ERR_INVALID_ARG;
-    if (d->dtype != FLARE_DTYPE_F32 && d->dtype != FLARE_DTYPE_BF16) return FLARE_ERR_UNSUPPORTED;
+    if (d->dtype != FLARE_DTYPE_F32 && d->dtype != FLARE_DTYPE_BF16 && d->dtype != FLARE_DTYPE_F16) return FLARE_ERR_UNSUPPORTED;
     if (d->D != 4 && d->D != 8 && d->D != 16 && d->D != 32 && d->D != 64) return FLARE_ERR_UNSUPPORTED;
     if (d->dtype == FLARE_DTYPE_BF16 && (d->M % 16 != 0 || d->M < 16 || d->M > 2048)) return FLARE_ERR_UNSUPPORTED;
     if ((long)d->B * d->N > (1L << 31) - 1 || d->H > 65535 || d->B > 65535) return FLARE_ERR_UNSUPPORTED;
@@ -789,8 +789,9 @@ int encode_impl(const flare_desc_t *d, const void *Q, const void *K, const void 
 #undef FLARE_ENC3
     } else {
         SimtPlan p = simt_plan(d, di.sms);
-        rc = (d->dtype == FLARE_DTYPE_F32) ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)
-                                           : launch_encode_simt<__nv_bfloat16>(d, p, Q, K, V, mask, pm, pl, pacc, st);
+        rc = (d->dtype == FLARE_DTYPE_F32)   ? launch_encode_simt<float>(d, p, Q, K, V, mask, pm, pl, pacc, st)
+             : (d->dtype == FLARE_DTYPE_F16) ? launch_encode_simt<__half>(d, p, Q, K, V, mask, pm, pl, pacc, st)
+                                             : launch_encode_simt<__nv_bfloat16>(d, p, Q, K, V, mask, pm, pl, pacc, st);
     }
     if (rc != FLARE_OK) return rc;
     if (P > 8)   // many partials (small problems spread over all SMs): a block per row shares the loads
@@ -851,8 +852,9 @@ int decode_impl(const flare_desc_t *d, const void *Q, const void *K, const float
             default: return decode_tc_any<64, 0>(d, sms, Q, K, Z, Y, lse_dec, status, range_scratch, st);
         }
     }
-    return (d->dtype == FLARE_DTYPE_F32) ? launch_decode_simt<float>(d, Q, K, Z, Y, lse_dec, st)
-                                         : launch_decode_simt<__nv_bfloat16>(d, Q, K, Z, Y, lse_dec, st);
+    return (d->dtype == FLARE_DTYPE_F32)   ? launch_decode_simt<float>(d, Q, K, Z, Y, lse_dec, st)
+           : (d->dtype == FLARE_DTYPE_F16) ? launch_decode_simt<__half>(d, Q, K, Z, Y, lse_dec, st)
+                                           : launch_decode_simt<__nv_bfloat16>(d, Q, K, Z, Y, lse_dec, st);
 }
 
 // Scratch of flare_encode_static_scratch: part of the device image, shared by every call on the device.
@@ -1012,6 +1014,8 @@ int expand_heads(const flare_desc_t *d, const void *src, void *dst, cudaStream_t
     const long per = (long)d->M * d->D, n = per * d->H;
     if (d->dtype == FLARE_DTYPE_F32)
         expand_heads_kernel<float><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const float *)src, (float *)dst, per, d->H);
+    else if (d->dtype == FLARE_DTYPE_F16)
+        expand_heads_kernel<__half><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const __half *)src, (__half *)dst, per, d->H);
     else
         expand_heads_kernel<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)src, (__nv_bfloat16 *)dst, per, d->H);
     FLARE_CUDA(cudaGetLastError());
@@ -1155,6 +1159,8 @@ int flare_backward(const flare_desc_t *desc, const void *Q_lat, const void *K, c
     cudaStream_t st = (cudaStream_t)stream;
     return desc->dtype == FLARE_DTYPE_F32
                ? backward_simt<float>(desc, sms, Q_lat, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ_lat, dK, dV, ws, st)
+           : desc->dtype == FLARE_DTYPE_F16
+               ? backward_simt<__half>(desc, sms, Q_lat, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ_lat, dK, dV, ws, st)
                : backward_simt<__nv_bfloat16>(desc, sms, Q_lat, K, V, key_mask, Y, dY, Z, lse_enc, lse_dec, dQ_lat, dK,
                                               dV, ws, st);
 }
@@ -1255,6 +1261,8 @@ int flare_backward_variant(const flare_desc_t *desc, int shared_latents, const v
     auto run = [&](const void *q, const float *le, const float *ld, float *dq, void *dk, bool skip_a) {
         return desc->dtype == FLARE_DTYPE_F32
                    ? backward_simt<float>(desc, sms, q, K, V, key_mask, Y, dY, Z, le, ld, dq, dk, dV, ws, st, skip_a)
+               : desc->dtype == FLARE_DTYPE_F16
+                   ? backward_simt<__half>(desc, sms, q, K, V, key_mask, Y, dY, Z, le, ld, dq, dk, dV, ws, st, skip_a)
                    : backward_simt<__nv_bfloat16>(desc, sms, q, K, V, key_mask, Y, dY, Z, le, ld, dq, dk, dV, ws, st, skip_a);
     };
     if (!separate) {
@@ -1274,6 +1282,8 @@ int flare_backward_variant(const flare_desc_t *desc, int shared_latents, const v
         const long nk = (long)desc->B * desc->N * desc->H * desc->D;
         if (desc->dtype == FLARE_DTYPE_F32)
             add_into_kernel<float><<<(unsigned)((nk + 255) / 256), 256, 0, st>>>((float *)dK, (const float *)dk2, nk);
+        else if (desc->dtype == FLARE_DTYPE_F16)
+            add_into_kernel<__half><<<(unsigned)((nk + 255) / 256), 256, 0, st>>>((__half *)dK, (const __half *)dk2, nk);
         else
             add_into_kernel<__nv_bfloat16><<<(unsigned)((nk + 255) / 256), 256, 0, st>>>((__nv_bfloat16 *)dK, (const __nv_bfloat16 *)dk2, nk);
         FLARE_CUDA(cudaGetLastError());
@@ -1303,8 +1313,9 @@ int flare_spectral_gram(const flare_desc_t *desc, const void *Q_lat, const void 
         return desc->D == 16 ? launch_spectral_gram_tc<16>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st)
                              : launch_spectral_gram_tc<32>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st);
     }
-    return desc->dtype == FLARE_DTYPE_F32 ? launch_spectral_gram_simt<float>(desc, Q_lat, K, lse_enc, lse_dec, G, st)
-                                          : launch_spectral_gram_simt<__nv_bfloat16>(desc, Q_lat, K, lse_enc, lse_dec, G, st);
+    return desc->dtype == FLARE_DTYPE_F32   ? launch_spectral_gram_simt<float>(desc, Q_lat, K, lse_enc, lse_dec, G, st)
+           : desc->dtype == FLARE_DTYPE_F16 ? launch_spectral_gram_simt<__half>(desc, Q_lat, K, lse_enc, lse_dec, G, st)
+                                            : launch_spectral_gram_simt<__nv_bfloat16>(desc, Q_lat, K, lse_enc, lse_dec, G, st);
 }
 
 int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues, float *U, int32_t sweeps, flare_stream_t stream) {

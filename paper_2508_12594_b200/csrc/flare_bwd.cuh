@@ -249,7 +249,7 @@ bwd_dq_simt_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__
             if (live) {
                 for (int j = g; j < kBwdTileN; j += G) {
                     float s0 = 0.f, a = 0.f, c = 0.f;
-                    if constexpr (std::is_same<T, float>::value) {
+                    if constexpr (!std::is_same<T, __nv_bfloat16>::value) {   // float32 and float16 inputs
                         double sd = 0.0;
 #pragma unroll
                         for (int d = 0; d < D; ++d) sd = fma((double)sQ[lm][d], (double)sK[j][d], sd);

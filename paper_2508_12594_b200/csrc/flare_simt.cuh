@@ -11,11 +11,11 @@
 
 namespace flare {
 
-// Score q.k of one (latent, token) pair.  For float32 inputs the products are summed in double so that the
-// score, which is exponentiated, carries no float32 summation error; bfloat16 inputs sum in float.
+// Score q.k of one (latent, token) pair.  For float32 and float16 inputs the products are summed in double so that
+// the score, which is exponentiated, carries no float32 summation error; bfloat16 inputs sum in float.
 template <typename T, int D>
 __device__ __forceinline__ float score_dot(const float (&a)[D], const float *b) {
-    if constexpr (std::is_same<T, float>::value) {
+    if constexpr (!std::is_same<T, __nv_bfloat16>::value) {   // float32 and float16 inputs
         double s = 0.0;
 #pragma unroll
         for (int d = 0; d < D; ++d) s = fma((double)a[d], (double)b[d], s);

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libflare.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(7)
-DTYPE_F32, DTYPE_BF16 = 0, 1
+DTYPE_F32, DTYPE_BF16, DTYPE_F16 = 0, 1, 2
 OP_ENCODE, OP_DECODE, OP_FORWARD, OP_BACKWARD, OP_SPECTRAL = range(5)
 
 
@@ -90,6 +90,8 @@ def _dtype_code(t: torch.Tensor) -> int:
         return DTYPE_F32
     if t.dtype == torch.bfloat16:
         return DTYPE_BF16
+    if t.dtype == torch.float16:
+        return DTYPE_F16
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 

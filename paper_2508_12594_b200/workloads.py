@@ -31,7 +31,7 @@ class Workload:
     N: int
     M: int
     D: int
-    dtype: str          # "f32" | "bf16"
+    dtype: str          # "f32" | "bf16" | "f16"
     kind: str           # "iid" | "cloud2d" | "padded" | "cube" | "scaled"
     seed: int
     backward: bool = False
@@ -42,7 +42,7 @@ class Workload:
         return self.B * self.N
 
     def torch_dtype(self) -> torch.dtype:
-        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+        return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[self.dtype]
 
     def with_(self, **kw) -> "Workload":
         return dataclasses.replace(self, **kw)
@@ -154,7 +154,7 @@ def make_random(B, H, N, M, D, dtype="f32", seed=0, masked_fraction=0.0, with_dy
     """Small i.i.d. Gaussian case for edge-shape tests; optional random padding mask."""
     g = torch.Generator(device="cpu")
     g.manual_seed(seed)
-    dt = torch.float32 if dtype == "f32" else torch.bfloat16
+    dt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[dtype]
     Q = (torch.randn(H, M, D, generator=g) * q_std).to(dt)
     K = (torch.randn(B, N, H, D, generator=g) * k_std).to(dt)
     V = torch.randn(B, N, H, D, generator=g).to(dt)

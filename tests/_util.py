@@ -7,7 +7,10 @@ from paper_2508_12594_b200 import flare
 
 # max |err| <= tol * RMS(reference), per tensor: 1e-5 for float32 inputs, 2e-2 for bfloat16 inputs with float32
 # accumulation (three bf16 roundings of relative size 2^-9 each: the softmax weights, Z and the stored Y).
-TOL = {"f32": 1e-5, "bf16": 2e-2}
+TOL = {"f32": 1e-5, "bf16": 2e-2, "f16": 2e-5}
+# float16 inputs run in float32 arithmetic (scores summed in double), so the float32 bound applies with a little room
+# for the float16 values' larger scores, plus one rounding of a stored float16 output (2^-11 |ref|, below).
+STORE_ULP = {"f32": 0.0, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}
 
 
 def rel_err(got, ref):
@@ -45,10 +48,10 @@ def assert_stored_close(got, ref, dtype, what):
     if plain <= tol:
         BOUND_LOG.append((what, "stated", plain, None))
         return "stated"
-    assert dtype == "bf16", f"{what}: max|err|/RMS = {plain:.3e} > {tol}"
-    excess = float((err - 2.0 ** -8 * np.abs(ref)).max()) / rms
+    assert dtype in ("bf16", "f16"), f"{what}: max|err|/RMS = {plain:.3e} > {tol}"
+    excess = float((err - STORE_ULP[dtype] * np.abs(ref)).max()) / rms
     BOUND_LOG.append((what, "stated+rounding", plain, excess))
-    assert excess <= tol, f"{what}: (max|err| - one bf16 rounding)/RMS = {excess:.3e} > {tol}"
+    assert excess <= tol, f"{what}: (max|err| - one rounding of the stored value)/RMS = {excess:.3e} > {tol}"
     return "stated+rounding"
 
 
@@ -115,4 +118,4 @@ def assert_forward_close(got, ref, dtype, what=""):
         assert np.array_equal(np.isneginf(got[name]), np.isneginf(ref[name])), f"{what} {name}: -inf pattern"
         if fin.any():
             err = np.abs(got[name][fin] - ref[name][fin]).max()
-            assert err <= (1e-4 if dtype == "f32" else 2e-2), f"{what} {name}: abs err {err:.3e}"
+            assert err <= (2e-2 if dtype == "bf16" else 1e-4), f"{what} {name}: abs err {err:.3e}"

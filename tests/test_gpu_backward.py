@@ -22,7 +22,7 @@ from tests._util import BOUND_LOG, dev, rel_err, to_np64
 
 pytestmark = pytest.mark.gpu
 
-GRAD_TOL = {"f32": 5e-5, "bf16": 2e-2}
+GRAD_TOL = {"f32": 5e-5, "bf16": 2e-2, "f16": 5e-5}
 
 
 def gpu_backward(inp, scale=1.0):
@@ -43,7 +43,7 @@ def assert_grads_close(got, ref, dtype, what, floor=None):
         rms = float(np.sqrt(np.mean(ref[name] ** 2)))
         if floor is not None:
             rms = max(rms, floor[name])
-        store_ulp = 2.0 ** -8 if (dtype == "bf16" and name != "dQ") else 0.0
+        store_ulp = 0.0 if name == "dQ" else {"f32": 0.0, "bf16": 2.0 ** -8, "f16": 2.0 ** -11}[dtype]
         err = np.abs(got[name] - ref[name])
         excess = err - store_ulp * np.abs(ref[name])
         e = float(excess.max()) / max(rms, 1e-300)
@@ -105,6 +105,10 @@ EDGE = [
     (1, 16, 500, 64, 4, "bf16", 0.0),
     (12, 16, 500, 144, 4, "bf16", 0.2),
     (1, 2, 200, 7, 4, "f32", 0.0),
+    # float16 inputs
+    (2, 3, 333, 48, 16, "f16", 0.3),
+    (1, 2, 400, 300, 32, "f16", 0.0),
+    (1, 4, 257, 7, 8, "f16", 0.0),
 ]
 
 

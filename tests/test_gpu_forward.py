@@ -82,6 +82,11 @@ EDGE = [
     (3, 2, 333, 5, 32, "f32", 0.4),
     (1, 1, 2049, 300, 64, "f32", 0.0),
     (1, 4, 64, 1, 16, "f32", 0.0),
+    # float16 inputs (the type the paper trains in): every entry point takes them, on the CUDA-core kernels
+    (2, 3, 333, 48, 16, "f16", 0.3),
+    (1, 2, 700, 300, 32, "f16", 0.0),
+    (1, 4, 257, 7, 8, "f16", 0.0),
+    (1, 2, 130, 64, 64, "f16", 0.2),
 ]
 
 
@@ -89,8 +94,8 @@ EDGE = [
 @STATS
 def test_edge_shapes(oracle, case, stats, path):
     B, H, N, M, D, dtype, mf = case
-    if dtype == "f32" and path == flare.PATH_FAST:
-        pytest.skip("float32 inputs run on the CUDA cores: one form only")
+    if dtype != "bf16" and path == flare.PATH_FAST:
+        pytest.skip("float32 and float16 inputs run on the CUDA cores: one form only")
     inp = workloads.make_random(B, H, N, M, D, dtype=dtype, seed=N + M, masked_fraction=mf, k_std=0.8)
     assert_forward_close(gpu_forward(inp, canary=True, stats=stats, path=path), oracle_forward(oracle, inp), dtype,
                          f"{case} {_mode(stats, path)}")

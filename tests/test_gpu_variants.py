@@ -21,6 +21,7 @@ CASES = [
     (1, 4, 900, 128, 32, "bf16", 0.0, True, True),
     (1, 2, 1300, 256, 16, "bf16", 0.1, True, True),
     (1, 8, 600, 64, 8, "bf16", 0.0, True, True),       # narrow heads
+    (2, 4, 500, 48, 16, "f16", 0.2, True, False),      # float16 inputs, one latent sequence for all heads
 ]
 
 
