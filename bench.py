@@ -32,8 +32,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) of one launch of each main kernel on the full mesh3d_1m workload, from the ncu captures
 # summarised under profiles/ (taken on a 262,144-token slice and scaled by 4: traffic is proportional to N).
 # Valid for the kernels as profiled; set to None when a kernel changes until the capture is redone.
-NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.328576e6 + 4.242176e6),     # profiles/encode_tc_fast_mesh3d_N262144.md
-               ("mesh3d_1m", "decode"): 4 * (67.379968e6 + 27.396352e6)}     # profiles/decode_stream_mesh3d_N262144.md
+NCU_TRAFFIC = {("mesh3d_1m", "encode"): 4 * (134.328320e6 + 5.408256e6),     # profiles/encode_tc_fast_mesh3d_N262144.md
+               ("mesh3d_1m", "decode"): 4 * (67.366912e6 + 26.701568e6)}     # profiles/decode_stream_mesh3d_N262144.md
 
 
 def get_workload(name: str) -> workloads.Workload:

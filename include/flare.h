@@ -252,7 +252,7 @@ int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues
  *   0, 1, 2   exponentials per clock per SM of the softmax loop as the sixteen softmax warps of a forward kernel run it
  *             (32 scores from tensor memory, 16 columns of packed weights back): 0 = with a running maximum and sum,
  *             special-function unit only; 1 = without a maximum, special-function unit only; 2 = without a maximum,
- *             every second pair of columns by the polynomial on the FMA pipe (what the fast forms run);
+ *             seven pairs of columns in sixteen by the polynomial on the FMA pipe (what the fast forms run);
  *   3, 4      cycles the issuing thread is held by one unit's tensor-core instructions (two value MMAs, one score MMA,
  *             one commit), and cycles from the commit to the flip of its barrier.
  * scratch: at least 4096 bytes of device memory.  *result is a HOST double.  Synchronises the stream.

@@ -10,7 +10,7 @@ namespace flare {
 
 // 16 warps (the softmax warps of the forward kernels) turn 32 score columns into 16 columns of packed weights, `iters` times.
 // kBody 0: running-maximum form (max, fma, ex2, sum, pack); 1: no maximum, special-function unit only; 2: no maximum,
-// every second pair of columns by the polynomial on the FMA pipe.  out[block] = cycles of the block's loop.
+// seven pairs of columns in sixteen (kPolyPairs) by the polynomial on the FMA pipe.  out[block] = cycles of the block's loop.
 template <int kBody>
 __global__ void __launch_bounds__(kTcThreads, 1) micro_softmax_kernel(int iters, float sl2, unsigned long long *out) {
     __shared__ uint32_t tmem_slot;

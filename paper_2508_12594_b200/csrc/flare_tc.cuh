@@ -186,8 +186,13 @@ constexpr float kFastMaxLog2 = 96.f;
 // rounded to bfloat16, 2e-3, right after), and adding round(x) to the exponent field is one shift-and-add on the
 // bits of t.  Valid for |x| < 126, which the fast forms guarantee; scores of padded tokens (kMaskedScore) must not
 // come this way.  Measured on B200 (16 warps, scores from and weights to tensor memory): 15 results per clock per SM
-// with the special-function unit alone, 24 with every second pair on the FMA pipe.
+// with the special-function unit alone, 22 with seven pairs in sixteen on the FMA pipe (see kPolyPairs; 24 with degree 2).
 constexpr int kPolyDegree = 3;
+// Which of every sixteen pairs of columns take the polynomial (bit k: pair k).  Measured, softmax loop alone /
+// million-point forward: 4 of 16: 19.0 exponentials per clock per SM / 1.195 ms; 5: 20.4 / 1.184; 6: 21.4 / 1.173;
+// 7: 22.3-22.5 / 1.128-1.155 (this pattern the better of two); 8 (every second pair): 21.4 / 1.161; 9: 20.6 / 1.269;
+// 10: 19.7 / 1.277.
+constexpr unsigned kPolyPairs = 0xAAA8;
 __device__ __forceinline__ float2 exp2_fma_pipe(float2 s, float2 sl2p) {
     constexpr float kMagic = 12582912.f;                        // 1.5 * 2^23
     const float2 magic = make_float2(kMagic, kMagic);
@@ -210,7 +215,7 @@ __device__ __forceinline__ float2 exp2_fma_pipe(float2 s, float2 sl2p) {
     return p;
 }
 
-// p = 2^(s * sl2) for NV scores, bf16 pairs to pk.  kPoly: every second pair on the FMA pipe.
+// p = 2^(s * sl2) for NV scores, bf16 pairs to pk.  kPoly: the pairs of kPolyPairs on the FMA pipe.
 // The row sum must be that of the ROUNDED weights: without a maximum the largest weight of a row is not 1.0 but
 // some 2^x with a full mantissa, and a sum of the unrounded values would normalise it away from the rounded one
 // that multiplies the values (measured: Y off by 1.5e-2 of its RMS where one weight dominates a row, against 4e-3).
@@ -225,7 +230,7 @@ __device__ __forceinline__ void exp_chunk_fast(const uint32_t *r, uint32_t *pk, 
     for (int k = 0; k < NV / 2; ++k) {
         const float2 s = make_float2(__uint_as_float(r[2 * k]), __uint_as_float(r[2 * k + 1]));
         float2 p;
-        if (kPoly && (k & 1)) {
+        if (kPoly && ((kPolyPairs >> (k & 15)) & 1)) {
             p = exp2_fma_pipe(s, sl2p);
         } else {
             const float2 x = __fmul2_rn(s, sl2p);
