@@ -1230,11 +1230,13 @@ struct EncodeSmem {
     static constexpr size_t kColBytes = 4 * kSoftmaxGroups * 2 * 32 * sizeof(float);   // per softmax warp: 2 x 32 column addends
     // score bias of padded tokens: per stage a [128 tokens, 16] bf16 tile, then one [128 latents, 16] tile of ones
     static constexpr size_t kBiasTile = kTile * 32;
+    // the tile of ones of the fast form exists only where its accumulator has room for the sum's column (DG + 16 <= 64)
+    static constexpr size_t kOnesBytes = DG + 16 <= 64 ? (size_t)kTile * G::RB : 0;
     static constexpr size_t total_for(int n) {
         size_t t = (size_t)n * 2 * G::TILE_BYTES + (size_t)2 * kTile * G::RB + 512 + kColBytes;
         t = (t + 1023) & ~(size_t)1023;
         t = (t + (size_t)(n + 1) * kBiasTile + 1023) & ~(size_t)1023;
-        return t + (size_t)kTile * G::RB + 1024;
+        return t + kOnesBytes + 1024;
     }
     static constexpr int stages_for() {
         int n = kAlt ? kEncMaxStages : kEncStages;
@@ -1250,7 +1252,7 @@ struct EncodeSmem {
     // fast form: a [128 tokens, DG] tile with a one in column 0 of every row, the value operand's second block along N
     __host__ __device__ static size_t ones_off() { return (bias_off() + (kStages + 1) * kBiasTile + 1023) & ~(size_t)1023; }
     __host__ __device__ static size_t total() {
-        size_t t = ones_off() + (size_t)kTile * G::RB + 1024;
+        size_t t = ones_off() + kOnesBytes + 1024;
         return t < kTcMinSmem ? kTcMinSmem : t;
     }
 };
