@@ -157,6 +157,57 @@ def run_micro():
     print(json.dumps({"micro": out}))
 
 
+def run_spectral(args, w):
+    """Algorithm 1 (spectral appendix) on the GPU for the workload's shape: the forward that yields the two log-sum-exp
+    arrays, the Gram matrix J J^T (one more pass over the tokens) and the M x M eigen-solver, each timed with CUDA events."""
+    from paper_2508_12594_b200 import flare
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    inp = workloads.make_inputs(w)
+    Q, K, V = inp.Q.cuda(), inp.K.cuda(), inp.V.cuda()
+    desc = flare.make_desc(Q, K, 1.0)
+    B, H, N, M, D = desc.B, desc.H, desc.N, desc.M, desc.D
+    ws, wss = flare.alloc_workspace(desc, flare.OP_FORWARD), flare.alloc_workspace(desc, flare.OP_SPECTRAL)
+    Y = torch.empty_like(K)
+    Z = torch.empty(B, H, M, D, dtype=torch.float32, device="cuda")
+    le = torch.empty(B, H, M, dtype=torch.float32, device="cuda")
+    ld = torch.empty(B, N, H, dtype=torch.float32, device="cuda")
+    G = torch.empty(B, H, M, M, dtype=torch.float32, device="cuda")
+    Gc, ev = torch.empty_like(G), torch.empty(B, H, M, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, steps):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(steps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / steps
+
+    steps = min(args.steps, 50)
+    t_fwd = timed(lambda: flare.flare_forward(desc, Q, K, V, None, Y, Z, le, ld, ws, stream), steps)
+    t_gram = timed(lambda: flare.flare_spectral_gram(desc, Q, K, le, ld, G, wss, stream), steps)
+
+    def eig():
+        Gc.copy_(G)
+        flare.flare_spectral_eig(Gc, ev, None, 0, stream)
+    t_eig = timed(eig, min(steps, 10))
+    flare.flare_check(wss)
+    top = float(ev[..., 0].mean())
+    peaks, kind = load_peaks()
+    flop = 2.0 * B * H * N * M * M                             # J J^T; the scores add 2 B H N M D
+    print(json.dumps({"spectral": {
+        "workload": w.name, "B": B, "H": H, "N": N, "M": M, "D": D, "dtype": w.dtype,
+        "forward_with_statistics_ms": t_fwd, "gram_ms": t_gram, "eig_ms": t_eig,
+        "gram_tflops": flop / (t_gram * 1e-3) / 1e12, "gram_frac_of_bf16_peak": flop / (t_gram * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "gram_bytes_gbs": (B * N * H * D * (2 if w.dtype != "f32" else 4) + 4.0 * B * N * H) / (t_gram * 1e-3) / 1e9,
+        "peak_kind": kind, "tokens_per_s": B * N / ((t_fwd + t_gram + t_eig) * 1e-3),
+        "largest_eigenvalue_mean": top}}))
+
+
 def run_reference(args, w):
     """The reference arm: the oracle on the host cores, each step a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -196,6 +247,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override N (a smaller case of the same workload)")
     ap.add_argument("--no-backward", action="store_true", help="skip the forward+backward leg")
     ap.add_argument("--micro", action="store_true", help="print the library's instruction-level measurements and exit")
+    ap.add_argument("--spectral", action="store_true",
+                    help="time the spectral analysis (Algorithm 1: forward statistics, Gram matrix, eigen-solver) on the workload and exit")
     args = ap.parse_args()
     w = get_workload(args.workload)
     if args.tokens > 0:
@@ -206,6 +259,8 @@ def main():
         return run_reference(args, w)
     if args.micro:
         return run_micro()
+    if args.spectral:
+        return run_spectral(args, w)
     if args.warmup < 3:
         args.warmup = 3
 

@@ -230,8 +230,9 @@ int flare_backward_variant(const flare_desc_t *desc, int shared_latents, const v
  * fix it as J J^T).  flare_spectral_gram forms G [B, H, M, M] float32 from Q_lat, K and the two log-sum-exp
  * outputs of flare_forward on the same Q_lat and K (lse_enc = log row sums, lse_dec = log column sums, both of
  * all tokens: no key mask), J[m,n] = exp(score - lse_enc[m]/2 - lse_dec[n]/2): one pass over the tokens, nothing of
- * size M x N is written.  bfloat16 inputs with M <= 128 and D in {16, 32} run on the tensor cores; everything else on
- * the CUDA cores.  Workspace: flare_workspace_bytes(desc, FLARE_OP_SPECTRAL).
+ * size M x N is written.  bfloat16 inputs with D in {16, 32} run on the tensor cores: M <= 128 in one pass, larger M
+ * (a multiple of 64, up to 1024) as one pass per pair of 64-latent blocks; everything else on the CUDA cores.
+ * Workspace: flare_workspace_bytes(desc, FLARE_OP_SPECTRAL).
  */
 int flare_spectral_gram(const flare_desc_t *desc, const void *Q_lat, const void *K, const float *lse_enc,
                         const float *lse_dec, float *G, void *workspace, size_t workspace_bytes, flare_stream_t stream);

@@ -1,6 +1,7 @@
 // Host side of libflare: argument checks, launch plans, kernel launches.  See include/flare.h for the contract.
 #include "../../include/flare.h"
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -910,7 +911,29 @@ int spectral_splits(const flare_desc_t *d, int sms) {
     if (s > tiles) s = tiles;
     return (int)s;
 }
+// More than 128 latents (a multiple of 64, bfloat16): the tensor-core kernel holds one block of 128 latents, so G is
+// assembled from runs over pairs of 64-latent blocks (i, j): the pair's rows of Q_lat and lse_enc are gathered into a
+// 128-latent problem, whose G holds the blocks G_ii, G_ij, G_ji, G_jj.  nb (nb - 1) / 2 runs, each one pass over the
+// tokens: 1.5 times the arithmetic of one pass over all latents, two orders of magnitude below the CUDA-core kernel.
+bool spectral_by_block_pairs(const flare_desc_t *d) {
+    return d->dtype == FLARE_DTYPE_BF16 && d->scale > 0.f && (d->D == 16 || d->D == 32) && d->M > kTile && d->M % 64 == 0 &&
+           d->M <= 1024;
+}
+struct SpectralPairLayout {
+    size_t part, qp, lep, gp, total;
+};
+SpectralPairLayout spectral_pair_layout(const flare_desc_t *d, int sms) {
+    SpectralPairLayout w{};
+    size_t off = kHeaderBytes;
+    w.part = off; off += align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * d->B * d->H * kTile * kTile);
+    w.qp = off;   off += align_up((size_t)d->H * kTile * d->D * 2);
+    w.lep = off;  off += align_up(sizeof(float) * (size_t)d->B * d->H * kTile);
+    w.gp = off;   off += align_up(sizeof(float) * (size_t)d->B * d->H * kTile * kTile);
+    w.total = off;
+    return w;
+}
 size_t spectral_bytes(const flare_desc_t *d, int sms) {
+    if (spectral_by_block_pairs(d) && use_tc(d)) return spectral_pair_layout(d, sms).total;
     if (!spectral_on_tensor_cores(d)) return kHeaderBytes;
     return kHeaderBytes + align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * d->B * d->H * kTile * kTile);
 }
@@ -938,6 +961,62 @@ int launch_spectral_gram_tc(const flare_desc_t *d, int sms, const void *Q, const
     const long n = (long)d->B * d->H * d->M * d->M;
     spectral_gram_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.part, G, a.splits, (long)d->B * d->H, d->M);
     FLARE_CUDA(cudaGetLastError());
+    return FLARE_OK;
+}
+
+// rows [64 i, 64 i + 64) and [64 j, 64 j + 64) of every head's Q_lat and lse_enc -> a 128-latent problem
+__global__ void spectral_gather_pair_kernel(const __nv_bfloat16 *__restrict__ Q, const float *__restrict__ lse_enc,
+                                            __nv_bfloat16 *__restrict__ Qp, float *__restrict__ lep, int B, int H, int M, int D,
+                                            int bi, int bj) {
+    const long t = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long nq = (long)H * kTile * D, nl = (long)B * H * kTile;
+    if (t < nq) {
+        const int dcol = (int)(t % D), r = (int)((t / D) % kTile), h = (int)(t / ((long)D * kTile));
+        const int m = 64 * (r < 64 ? bi : bj) + (r & 63);
+        Qp[t] = Q[((size_t)h * M + m) * D + dcol];
+    }
+    if (t < nl) {
+        const int r = (int)(t % kTile);
+        const long bh = t / kTile;
+        lep[t] = lse_enc[bh * M + 64 * (r < 64 ? bi : bj) + (r & 63)];
+    }
+}
+// the pair's [128, 128] result -> the blocks (i, j), (j, i) of G, and the diagonal blocks this pair is responsible for
+__global__ void spectral_scatter_pair_kernel(const float *__restrict__ Gp, float *__restrict__ G, long BH, int M, int bi, int bj,
+                                             int write_ii, int write_jj) {
+    const long t = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= BH * kTile * kTile) return;
+    const int c = (int)(t % kTile), r = (int)((t / kTile) % kTile);
+    const long bh = t / ((long)kTile * kTile);
+    const bool rj = r >= 64, cj = c >= 64;
+    if (!rj && !cj && !write_ii) return;
+    if (rj && cj && !write_jj) return;
+    G[(bh * M + 64 * (rj ? bj : bi) + (r & 63)) * M + 64 * (cj ? bj : bi) + (c & 63)] = Gp[t];
+}
+
+template <int D>
+int spectral_gram_block_pairs(const flare_desc_t *d, int sms, const void *Q, const void *K, const float *lse_enc,
+                              const float *lse_dec, float *G, char *ws, cudaStream_t st) {
+    const SpectralPairLayout w = spectral_pair_layout(d, sms);
+    __nv_bfloat16 *Qp = reinterpret_cast<__nv_bfloat16 *>(ws + w.qp);
+    float *lep = reinterpret_cast<float *>(ws + w.lep), *Gp = reinterpret_cast<float *>(ws + w.gp);
+    flare_desc_t dp = *d;
+    dp.M = kTile;
+    const int nb = d->M / 64;
+    const long BH = (long)d->B * d->H;
+    const long ngather = std::max((long)d->H * kTile * d->D, BH * kTile), nscatter = BH * kTile * kTile;
+    for (int i = 0; i < nb; ++i)
+        for (int j = i + 1; j < nb; ++j) {
+            spectral_gather_pair_kernel<<<(unsigned)((ngather + 255) / 256), 256, 0, st>>>(
+                static_cast<const __nv_bfloat16 *>(Q), lse_enc, Qp, lep, d->B, d->H, d->M, d->D, i, j);
+            FLARE_CUDA(cudaGetLastError());
+            const int rc = launch_spectral_gram_tc<D>(&dp, sms, Qp, K, lep, lse_dec, Gp, ws, st);
+            if (rc != FLARE_OK) return rc;
+            // every diagonal block is written once: G_ii by the pair (i, i + 1), the last one by the last pair
+            spectral_scatter_pair_kernel<<<(unsigned)((nscatter + 255) / 256), 256, 0, st>>>(
+                Gp, G, BH, d->M, i, j, j == i + 1, (i == nb - 2 && j == nb - 1) ? 1 : 0);
+            FLARE_CUDA(cudaGetLastError());
+        }
     return FLARE_OK;
 }
 
@@ -1308,6 +1387,11 @@ int flare_spectral_gram(const flare_desc_t *desc, const void *Q_lat, const void 
     if (workspace_bytes < spectral_bytes(desc, sms)) return FLARE_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     FLARE_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, st));
+    if (spectral_by_block_pairs(desc) && use_tc(desc)) {
+        char *ws = static_cast<char *>(workspace);
+        return desc->D == 16 ? spectral_gram_block_pairs<16>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st)
+                             : spectral_gram_block_pairs<32>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st);
+    }
     if (spectral_on_tensor_cores(desc) && use_tc(desc)) {
         char *ws = static_cast<char *>(workspace);
         return desc->D == 16 ? launch_spectral_gram_tc<16>(desc, sms, Q_lat, K, lse_enc, lse_dec, G, ws, st)
@@ -1326,7 +1410,9 @@ int flare_spectral_eig(int32_t matrices, int32_t M, float *G, float *eigenvalues
     if (sweeps <= 0) sweeps = 12;
     const int pairs = ((M + 1) & ~1) / 2;
     const size_t shmem = sizeof(float) * (4 * (size_t)pairs + M);
-    spectral_jacobi_kernel<<<(unsigned)matrices, 256, shmem, (cudaStream_t)stream>>>(G, eigenvalues, U, M, sweeps);
+    // a step's rotations touch pairs * M elements: one thread each up to the largest block (the steps are latency-bound)
+    const int threads = M >= 128 ? 1024 : M >= 64 ? 512 : 256;
+    spectral_jacobi_kernel<<<(unsigned)matrices, threads, shmem, (cudaStream_t)stream>>>(G, eigenvalues, U, M, sweeps);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }

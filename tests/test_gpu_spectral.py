@@ -19,10 +19,11 @@ CASES = [
     (1, 2, 1024, 16, 16, "f32", 1.0),        # the tiny configuration's shape: CUDA cores
     (2, 2, 972, 64, 16, "bf16", 1.0),        # the paper's spectra are of N = 972, M = 64: one latent block on the tensor cores
     (1, 2, 3001, 128, 16, "bf16", 0.7),      # all 128 lanes, several tiles, a ragged tail
-    (1, 2, 1300, 256, 16, "bf16", 0.7),      # more than 128 latents: CUDA cores
+    (1, 2, 1300, 256, 16, "bf16", 0.7),      # more than 128 latents, a multiple of 64: pairs of 64-latent blocks on the tensor cores
+    (2, 2, 900, 192, 32, "bf16", 0.6),       # three blocks
     (1, 4, 1500, 128, 32, "bf16", 0.5),
     (1, 2, 700, 48, 32, "bf16", 1.0),        # a latent block that is mostly empty lanes
-    (1, 2, 600, 400, 16, "bf16", 0.5),
+    (1, 2, 600, 400, 16, "bf16", 0.5),       # not a multiple of 64: CUDA cores
     (1, 2, 500, 32, 8, "bf16", 1.0),         # narrow heads: CUDA cores
 ]
 
