@@ -925,7 +925,7 @@ struct SpectralPairLayout {
 SpectralPairLayout spectral_pair_layout(const flare_desc_t *d, int sms) {
     SpectralPairLayout w{};
     size_t off = kHeaderBytes;
-    w.part = off; off += align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * d->B * d->H * kTile * kTile);
+    w.part = off; off += align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * kSpectralGroups * d->B * d->H * kTile * kTile);
     w.qp = off;   off += align_up((size_t)d->H * kTile * d->D * 2);
     w.lep = off;  off += align_up(sizeof(float) * (size_t)d->B * d->H * kTile);
     w.gp = off;   off += align_up(sizeof(float) * (size_t)d->B * d->H * kTile * kTile);
@@ -935,7 +935,7 @@ SpectralPairLayout spectral_pair_layout(const flare_desc_t *d, int sms) {
 size_t spectral_bytes(const flare_desc_t *d, int sms) {
     if (spectral_by_block_pairs(d) && use_tc(d)) return spectral_pair_layout(d, sms).total;
     if (!spectral_on_tensor_cores(d)) return kHeaderBytes;
-    return kHeaderBytes + align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * d->B * d->H * kTile * kTile);
+    return kHeaderBytes + align_up(sizeof(float) * (size_t)spectral_splits(d, sms) * kSpectralGroups * d->B * d->H * kTile * kTile);
 }
 
 template <int D>
@@ -959,7 +959,7 @@ int launch_spectral_gram_tc(const flare_desc_t *d, int sms, const void *Q, const
     spectral_gram_tc_kernel<D><<<dim3(a.splits, d->H, d->B), kTcThreads, SpectralSmem<D>::total, st>>>(tmK, tmQ, a);
     FLARE_CUDA(cudaGetLastError());
     const long n = (long)d->B * d->H * d->M * d->M;
-    spectral_gram_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.part, G, a.splits, (long)d->B * d->H, d->M);
+    spectral_gram_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.part, G, a.splits * kSpectralGroups, (long)d->B * d->H, d->M);
     FLARE_CUDA(cudaGetLastError());
     return FLARE_OK;
 }

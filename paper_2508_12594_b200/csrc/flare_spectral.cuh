@@ -30,27 +30,32 @@ struct SpectralArgs {
     const __nv_bfloat16 *Q;   // [H,M,D]
     const float *lse_enc;     // [B,H,M]
     const float *lse_dec;     // [B,N,H]
-    float *part;              // [splits][B*H][128][128] float32 partial sums of G
+    float *part;              // [splits * kSpectralGroups][B*H][128][128] float32 partial sums of G
     uint32_t *status;
     int B, H, N, M;
     float sl2;                // scale * log2(e)
     int tiles, splits;
 };
 
+// Groups of 128 threads at work in a CTA of the tensor-core Gram kernel: each takes every third token tile with its own
+// score buffer, accumulator (160 of the 512 tensor-memory columns) and partial sum.
+constexpr int kSpectralGroups = 3;
+
 template <int D>
 struct SpectralSmem {
     using G = TileGeom<D>;
-    static constexpr int kStages = 3;
+    static constexpr int kStages = 6;
     static constexpr size_t k_off = 0;                                      // K tiles
     static constexpr size_t q_off = (size_t)kStages * G::TILE_BYTES;        // Q rows
     static constexpr size_t pb_off = q_off + (size_t)kTile * G::RB;         // J (hi, lo) as B operands: [128 latents, 32 tokens] bf16 each
     static constexpr size_t kPbBytes = (size_t)kTile * 64;
-    static constexpr size_t col_off = pb_off + 2 * kPbBytes;                // per softmax warp 32 column addends
-    static constexpr size_t bar_off = (col_off + 4 * 32 * sizeof(float) + 1023) & ~(size_t)1023;
+    static constexpr size_t col_off = pb_off + kSpectralGroups * 2 * kPbBytes;   // (a hi and a lo tile per group); per softmax warp 32 column addends
+    static constexpr size_t bar_off = (col_off + kSpectralGroups * 4 * 32 * sizeof(float) + 1023) & ~(size_t)1023;
     static constexpr size_t total = bar_off + 512 + 1024 < kTcMinSmem ? kTcMinSmem : bar_off + 512 + 1024;
 };
 
-// grid = (splits, H, B).  Warp 0: TMA; warp 1: MMA issue; warps 5-8: the 128 threads of the latent rows.
+// grid = (splits, H, B).  Warp 0: TMA; warps 1-3: MMA issue, one per group; warps 5-16: three groups of 128 threads, the
+// latent rows on their lanes.  Group g works on the tiles g, g + 3, ... of the CTA's range and leaves its own partial sum.
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 spectral_gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ, SpectralArgs a) {
@@ -63,11 +68,13 @@ spectral_gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     float *colneg = reinterpret_cast<float *>(smem + SM::col_off);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM::bar_off);
     constexpr int kStages = SM::kStages, UNIT = 32;
-    enum { K_FULL = 0, K_EMPTY = K_FULL + kStages, Q_FULL = K_EMPTY + kStages, S_FULL, P_FULL, G_DONE, NBARS };
+    constexpr int NGS = kSpectralGroups;
+    enum { K_FULL = 0, K_EMPTY = K_FULL + kStages, Q_FULL = K_EMPTY + kStages, S_FULL, P_FULL = S_FULL + NGS,
+           G_DONE = P_FULL + NGS, NBARS = G_DONE + NGS };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + NBARS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
-    // tensor memory: G [0,128)  S [128,160)
-    constexpr uint32_t G_AA = 0, S_A = 128, NCOLS = 256;
+    // tensor memory, per group 160 columns: G [0,128)  S [128,160)
+    constexpr uint32_t G_AA = 0, S_A = 128, GROUP_COLS = 160, NCOLS = 512;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -77,7 +84,7 @@ spectral_gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     auto bar = [&](int i) { return ptx::smem_u32(bars + i); };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NBARS; ++i) ptx::mbar_init(bar(i), i == P_FULL ? 4u : 1u);   // P_FULL: one arrival per warp
+        for (int i = 0; i < NBARS; ++i) ptx::mbar_init(bar(i), (i >= P_FULL && i < P_FULL + NGS) ? 4u : 1u);   // P_FULL: one arrival per warp
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmK);
@@ -103,28 +110,31 @@ spectral_gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
                 ptx::tma_load_3d(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), &tmK, bar(K_FULL + s), h * D, (t_begin + i) * kTile, b);
             }
         }
-    } else if (warp == kFirstIssuerWarp) {
+    } else if (warp >= kFirstIssuerWarp && warp < kFirstIssuerWarp + NGS) {
+        const int g = warp - kFirstIssuerWarp;
+        const int mytiles = (nt - g + NGS - 1) / NGS;
+        const uint32_t gtm = tm + g * GROUP_COLS;
         if (lane == 0) {
             const uint32_t idescS = ptx::instr_desc_bf16(128, UNIT, 0, 0), idescG = ptx::instr_desc_bf16(128, 128, 0, 0);
             const uint64_t qdesc = ptx::smem_desc(ptx::smem_u32(sQ), 16, G::SBO, G::SWZ);
-            const uint64_t pbdesc = ptx::smem_desc(ptx::smem_u32(sPB), 16, GP::SBO, GP::SWZ);
+            const uint64_t pbdesc = ptx::smem_desc(ptx::smem_u32(sPB + (size_t)g * 2 * SM::kPbBytes), 16, GP::SBO, GP::SWZ);
             bool ok = ptx::mbar_wait(bar(Q_FULL), 0, abort_flag, kErrSpectral | 2);
-            const int units = 4 * nt;
-            auto issue_scores = [&](int u) -> bool {              // unit u: tile u / 4, tokens 32 (u % 4) ... of it
-                const int i = u >> 2, s = i % kStages;
+            const int units = 4 * mytiles;
+            auto issue_scores = [&](int u) -> bool {              // unit u: the group's tile u / 4, tokens 32 (u % 4) ... of it
+                const int i = g + NGS * (u >> 2), s = i % kStages;
                 if ((u & 3) == 0 && !ptx::mbar_wait(bar(K_FULL + s), (i / kStages) & 1, abort_flag, kErrSpectral | 3)) return false;
                 ptx::tc_fence_after();
                 const uint64_t kdesc = ptx::smem_desc(ptx::smem_u32(sK + (size_t)s * G::TILE_BYTES), 16, G::SBO, G::SWZ) +
                                        (uint64_t)(((u & 3) * UNIT * G::RB) >> 4);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(tm + S_A, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
-                ptx::mma_commit(bar(S_FULL));
+                for (int k = 0; k < D / 16; ++k) ptx::mma_ss(gtm + S_A, qdesc + 2 * k, kdesc + 2 * k, idescS, k > 0);
+                ptx::mma_commit(bar(S_FULL + g));
                 if ((u & 3) == 3) ptx::mma_commit(bar(K_EMPTY + s));
                 return true;
             };
             if (ok && units > 0) ok = issue_scores(0);
             for (int u = 0; ok && u < units; ++u) {
-                if (!ptx::mbar_wait(bar(P_FULL), u & 1, abort_flag, kErrSpectral | 4)) break;
+                if (!ptx::mbar_wait(bar(P_FULL + g), u & 1, abort_flag, kErrSpectral | 4)) break;
                 ptx::tc_fence_after();
                 // G += J J^T over the unit's 32 tokens (two k-steps of 16): A = J in tensor memory (hi in the first 16 columns
                 // of the score buffer, lo in the other 16), B = J in shared memory (hi tile, then lo tile)
@@ -136,32 +146,34 @@ spectral_gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
                         const uint32_t acol = (t == 2 ? 16u : 0u) + 8 * k;
                         const uint64_t bsel = (t == 1 ? LO : 0) + 2 * k;
                         const uint32_t acc = (u > 0 || k > 0 || t > 0) ? 1u : 0u;
-                        ptx::mma_ts(tm + G_AA, tm + S_A + acol, pbdesc + bsel, idescG, acc);
+                        ptx::mma_ts(gtm + G_AA, gtm + S_A + acol, pbdesc + bsel, idescG, acc);
                     }
                 }
                 // the next unit's scores overwrite J in tensor memory after those MMAs (a thread's MMAs run in order); the
                 // commit behind them also tells the threads that J in shared memory has been read
                 if (u + 1 < units) ok = issue_scores(u + 1);
-                else ptx::mma_commit(bar(G_DONE));
+                else ptx::mma_commit(bar(G_DONE + g));
             }
         }
-    } else if (warp >= kFirstSoftmaxWarp && warp < kFirstSoftmaxWarp + 4) {
+    } else if (warp >= kFirstSoftmaxWarp && warp < kFirstSoftmaxWarp + 4 * NGS) {
+        const int g = (warp - kFirstSoftmaxWarp) >> 2;
+        const int mytiles = (nt - g + NGS - 1) / NGS;
         const int row = ((warp & 3) << 5) + lane;               // TMEM lane = latent
         const int m = row;
         const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
-        const uint32_t scol = tm + lane_addr + S_A;
+        const uint32_t scol = tm + lane_addr + g * GROUP_COLS + S_A;
         float *cn = colneg + (warp - kFirstSoftmaxWarp) * 32;
         const float rowneg = m < M ? -0.5f * 1.4426950408889634f * a.lse_enc[((size_t)b * a.H + h) * M + m] : -INFINITY;
         const float2 sl2p = make_float2(a.sl2, a.sl2);
-        uint8_t *pb = sPB + (size_t)row * GP::RB;               // this latent's row of the hi tile; lo: kPbBytes on
+        uint8_t *pb = sPB + (size_t)g * 2 * SM::kPbBytes + (size_t)row * GP::RB;   // this latent's row of the group's hi tile; lo: kPbBytes on
         bool ok = true;
-        const int units = 4 * nt;
+        const int units = 4 * mytiles;
         for (int u = 0; ok && u < units; ++u) {
-            const int n = (t_begin + (u >> 2)) * kTile + (u & 3) * UNIT + lane;     // this lane fetches the shift of token n
+            const int n = (t_begin + g + NGS * (u >> 2)) * kTile + (u & 3) * UNIT + lane;   // this lane fetches the shift of token n
             __syncwarp();
             cn[lane] = n < a.N ? -0.5f * 1.4426950408889634f * a.lse_dec[((size_t)b * a.N + n) * a.H + h] : -INFINITY;
             __syncwarp();
-            if (!(ok = warp_wait(bar(S_FULL), u & 1, abort_flag, kErrSpectral | 5))) break;
+            if (!(ok = warp_wait(bar(S_FULL + g), u & 1, abort_flag, kErrSpectral | 5))) break;
             ptx::tc_fence_after();
             uint32_t r[32], hi[16], lo[16];
             ptx::tmem_ld32(scol, r);
@@ -192,18 +204,18 @@ spectral_gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             ptx::tmem_wait_st();
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(P_FULL));
+            if (lane == 0) ptx::mbar_arrive(bar(P_FULL + g));
         }
         // the partial sum of G: this thread's lane holds row m
-        if (ok && units > 0) ok = warp_wait(bar(G_DONE), 0, abort_flag, kErrSpectral | 6);
+        if (ok && units > 0) ok = warp_wait(bar(G_DONE + g), 0, abort_flag, kErrSpectral | 6);
         ptx::tc_fence_after();
         if (ok) {
-            float *dst = a.part + (((size_t)split * a.B + b) * a.H + h) * (size_t)kTile * kTile + (size_t)row * kTile;
+            float *dst = a.part + ((((size_t)split * NGS + g) * a.B + b) * a.H + h) * (size_t)kTile * kTile + (size_t)row * kTile;
 #pragma unroll 1
             for (int c0 = 0; c0 < kTile; c0 += 32) {
                 uint32_t v[32];
                 if (units > 0) {
-                    ptx::tmem_ld32(tm + lane_addr + G_AA + c0, v);
+                    ptx::tmem_ld32(tm + lane_addr + g * GROUP_COLS + G_AA + c0, v);
                     ptx::tmem_wait_ld();
                 } else {
 #pragma unroll
