@@ -333,9 +333,11 @@ spectral_jacobi_kernel(float *__restrict__ Gall, float *__restrict__ evals, floa
                 cs[k] = c; cs[pairs + k] = s; pp[k] = p; pp[pairs + k] = q;
             }
             __syncthreads();
-            // columns: G <- G R (and U <- U R), every row independently
+            // columns: G <- G R (and U <- U R), every row independently.  Neighbouring threads take the pairs of one row:
+            // a step's pairs cover every column once, so the row's sectors are all used while they are in the cache
+            // (pair-major order touched one element per sector and was 3 times slower at M = 512).
             for (int i = t; i < pairs * M; i += T) {
-                const int k = i / M, row = i % M, p = pp[k], q = pp[pairs + k];
+                const int row = i / pairs, k = i % pairs, p = pp[k], q = pp[pairs + k];
                 if (q >= M) continue;
                 const float c = cs[k], s = cs[pairs + k];
                 const float gp = G[(size_t)row * M + p], gq = G[(size_t)row * M + q];
