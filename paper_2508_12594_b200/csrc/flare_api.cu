@@ -146,12 +146,14 @@ bool use_fast(const flare_desc_t *d, FastStage stage) {
     if (path == FLARE_PATH_EXACT) return false;
     if (path == FLARE_PATH_FAST) return true;
     // Measured (forward stage times, fast against exact form): encode wins from 128 latents (3-5 % there, 15 % at 256),
-    // loses at 32 and 64 latents of width 32; the streaming decode
+    // is equal or loses at 32 and 64 latents of width 32; the streaming decode
     // wins from 64 latents (16 % at 64 and 128) and loses at 32; below some tens of microseconds of work the two extra
     // launches cost more than the forms gain.
-    // (The head-pair form of encode, M <= 64, neither wins nor loses at D = 16 and loses at D = 32, where it has no room
-    // for the ones column and sums the weights in registers.)
-    const bool big_enough = d->M >= (stage == kFastEncode ? 128 : 64);
+    // The head-pair form of encode (M <= 64, H even) wins at D = 16 since its K/V ring is deep (0.077 -> 0.062 ms on the
+    // 2-D mesh: its rows are short scans, in which the exact form rescales its accumulator on most units) and is equal
+    // at D = 32, where it has no room for the ones column and sums the weights in registers.
+    const bool pair16 = d->M <= 64 && d->H % 2 == 0 && d->D == 16;
+    const bool big_enough = stage == kFastEncode ? (d->M >= 128 || pair16) : d->M >= 64;
     return big_enough && (double)d->B * d->H * d->N * d->M >= 3.0e7;
 }
 
